@@ -1,0 +1,181 @@
+/*
+ * rptq.h -- C boundary of the B200 (sm_100a) library for the hot path of RPTQ, reorder-based
+ * post-training quantisation (arXiv 2304.01089).
+ *
+ * The library holds two device kernels and the small amount of host logic around them:
+ *
+ *   rptq_ln_reorder_quant   LayerNorm -> channel reorder -> per-cluster quantise -> packed codes
+ *   rptq_cluster_gemm       packed activation codes x packed int4 weights, integer products per
+ *                           cluster segment on the tensor cores, floating-point epilogue
+ *
+ * Conventions
+ *   - Every function returns an int status: RPTQ_OK or a negative RPTQ_ERR_* value. Nothing
+ *     throws, aborts or prints.
+ *   - "dev" pointers are device global memory of the device that was current when the layout
+ *     was created; "host" pointers are ordinary host memory. The caller owns every buffer. The
+ *     library allocates device memory only inside rptq_layout_create (small tables) and for one
+ *     lazily created status word per process.
+ *   - Kernel launches are asynchronous on `stream` (a cudaStream_t passed as void*; NULL is the
+ *     default stream). A layout handle is immutable after creation and may be used from several
+ *     streams at once.
+ *   - dev pointers must be 16-byte aligned.
+ *
+ * Notation (paper, Sec. 4.1 and Appendix "Computation under cluster-based quantization"):
+ *   M tokens, C channels, g clusters, k (here `bits`) activation bits, N output channels,
+ *   S = [S^1 .. S^g] the reorder index, n_c = |S^c|, (s_c, z_c) the quantisation parameters of
+ *   cluster c.
+ *
+ * Padded segment layout (not in the paper; the tensor-core contraction step is 32 codes wide and
+ * operands are staged in blocks of 128): in a row of codes cluster c occupies positions
+ * seg_off[c] .. seg_off[c] + n_c - 1 with seg_off[c] = sum_{c' < c} roundup32(n_c'), and the row
+ * length is K_pad = max(128, roundup128(seg_off[g])). Pad positions hold activation code 0 and
+ * weight code 0.
+ *
+ * Packed storage, format version 1 (private to this library; read it back with the *_unpack_host
+ * helpers). A row of K_pad codes takes K_pad*bits/8 bytes:
+ *   8 bit  one byte per code;
+ *   4 bit  32-bit little-endian word w holds codes 8w..8w+7: byte i (0..3) carries code 8w+i in
+ *          bits 0-3 and code 8w+4+i in bits 4-7;
+ *   3 bit  32 codes take three words; word j carries codes 8j..8j+7 of the group as in the 4-bit
+ *          layout, and bit 3 of nibble t of word j carries bit j of code 24+t (nibble t = low
+ *          nibble of byte t for t < 4, high nibble of byte t-4 otherwise).
+ * Weight codes are signed 4-bit two's-complement nibbles in the 4-bit layout.
+ */
+#ifndef RPTQ_H_
+#define RPTQ_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    RPTQ_OK = 0,
+    RPTQ_ERR_INVALID_ARG = -1,     /* null pointer, negative size, misaligned pointer, bad stride */
+    RPTQ_ERR_UNSUPPORTED = -2,     /* a size or option outside what the kernels handle */
+    RPTQ_ERR_NOT_BIJECTION = -3,   /* perm is not a permutation of 0..C-1, or sizes do not sum to C */
+    RPTQ_ERR_CUDA = -4,            /* a CUDA runtime or driver call failed */
+    RPTQ_ERR_DEVICE_TIMEOUT = -5,  /* a bounded wait inside a kernel ran out (see rptq_get_device_status) */
+    RPTQ_ERR_ALLOC = -6            /* host or device allocation failed */
+};
+
+enum { RPTQ_OUT_F32 = 0, RPTQ_OUT_F16 = 1, RPTQ_OUT_CODES = 2 };
+enum { RPTQ_ACT_NONE = 0, RPTQ_ACT_RELU = 1 };
+enum { RPTQ_FORMAT_VERSION = 1 };
+
+typedef struct rptq_layout rptq_layout_t;
+
+/*
+ * Sec. 4.1: the reorder index S (concatenated cluster index sets) with one (s_c, z_c) per
+ * cluster (Sec. 5.1: per-cluster asymmetric parameters), for a site with C channels quantised
+ * to `bits` in {3, 4, 8}.
+ *   perm_host[C]     S: reordered position j holds original channel perm_host[j]; must be a
+ *                    permutation of 0..C-1 (else RPTQ_ERR_NOT_BIJECTION).
+ *   cluster_size[g]  n_c >= 0 in the order the clusters appear in S; must sum to C.
+ *   scale_host[g]    s_c > 0 and finite.
+ *   zero_host[g]     z_c for codes re-based to [0, 2^bits - 1] (Eq. 1 states the signed range
+ *                    [-2^(k-1), 2^(k-1)-1]; adding 2^(k-1) to both code and zero point leaves
+ *                    s (x_q - z) unchanged). |z_c| < 2^21.
+ * Limits: C a multiple of 8, 8 <= C <= 65528, 1 <= g <= 4096, K_pad <= 65408; otherwise
+ * RPTQ_ERR_UNSUPPORTED. On success *out owns small device tables on the current device; free it
+ * with rptq_layout_destroy. All four arrays are copied.
+ */
+int rptq_layout_create(rptq_layout_t** out, int C, int g, int bits,
+                       const int32_t* perm_host, const int32_t* cluster_size,
+                       const float* scale_host, const int32_t* zero_host);
+
+/* Sizes of the padded layout. Any output pointer may be NULL. seg_offset_out receives g+1 ints. */
+int rptq_layout_query(const rptq_layout_t* L, int* K_pad, int64_t* row_bytes, int32_t* seg_offset_out);
+
+/* Frees the handle and its device tables. Work that uses it must have completed. NULL is OK. */
+int rptq_layout_destroy(rptq_layout_t* L);
+
+/*
+ * Sec. 4.2 "we fuse the reorder operation into the layer norm operation", followed by the
+ * cluster quantiser of the Appendix, X~_q,c = Q_k(X~_c, s_c, z_c) with Q_k of Eq. 1:
+ *   mu = mean_c x[m][c], var = mean_c (x[m][c]-mu)^2, y[c] = (x[m][c]-mu)/sqrt(var+eps)*gamma[c]+beta[c]
+ *   (fp32 arithmetic on fp16 inputs), then for reordered position j in cluster c
+ *   q = clamp(rne(y[S_j] / s_c) + z_c, 0, 2^bits - 1)
+ * where y / s_c is evaluated as the exact product of y (fp32) and the fp32 reciprocal
+ * (float)(1.0/(double)s_c), rounded once, half to even, to an integer.
+ *   x      dev fp16 [M][ldx], ldx >= C, ldx a multiple of 8
+ *   gamma  dev fp16 [C], beta dev fp16 [C]  (original channel order)
+ *   codes  dev, M rows of row_bytes bytes, packed as described above; every byte is written
+ *   y_dbg  NULL, or dev fp32 [M][C]: receives the LayerNorm outputs in reordered channel order
+ *          (the values the codes were decided from)
+ * M >= 0 (M == 0 launches nothing). Non-finite inputs give in-range codes, not an error.
+ */
+int rptq_ln_reorder_quant(const rptq_layout_t* L, const void* x, int64_t ldx, const void* gamma,
+                          const void* beta, float eps, int M, void* codes, float* y_dbg, void* stream);
+
+/*
+ * Sec. 4.2: "We reorder the columns of the weight matrix (dimension C1) based on the input
+ * activation reorder index, and the rows (dimension C2) based on the output activation reorder
+ * index"; done once before deployment, on the host. W_host is fp32 [N][C] in the [out][in]
+ * orientation (Y = X W^T). Weights are quantised round-to-nearest, symmetric, one scale per output
+ * channel (the paper uses GPTQ, which needs a trained model's statistics):
+ *   s_w[n] = max_k |W[n][k]| / 7 (1 if the row is zero), w_q = clamp(rne(W / s_w), -8, 7), in fp32.
+ *   out_perm      NULL, or host int32 [N]: output row r is original row out_perm[r]
+ *   N_pad         >= N; rows N..N_pad-1 are zero with s_w = 1
+ *   w_codes_host  host, N_pad rows of K_pad/2 bytes (packed signed nibbles, padded segment layout)
+ *   s_w           host fp32 [N_pad]
+ *   wsum          host int32 [g][N_pad]: Wsum_c[r] = sum of w_q over the channels of cluster c
+ * Runs on the calling thread plus OpenMP workers; touches no device.
+ */
+int rptq_weight_pack(const rptq_layout_t* Lin, const float* W_host, int N, const int32_t* out_perm,
+                     int N_pad, void* w_codes_host, float* s_w, int32_t* wsum);
+
+/*
+ * Appendix, second computation method, with symmetric per-output-channel weights (z^W = 0):
+ *   acc_c[m][n] = sum_{k in segment c} X_q[m][k] * W_q[n][k]                (int32, exact)
+ *   y[m][n]     = s_w[n] * sum_c s_c * (acc_c[m][n] - z_c * Wsum_c[n])  (+ bias[n]) (ReLU)
+ * in fp32, optionally re-quantised for the next layer (Sec. 4.2: the output channel order is
+ * that of the weight's rows, so a following reordered site reads it without an explicit reorder).
+ *   a_codes  dev, M rows of Lin.row_bytes bytes (as written by rptq_ln_reorder_quant or by this
+ *            function with RPTQ_OUT_CODES)
+ *   w_codes  dev, N_pad rows of Lin.K_pad/2 bytes; s_w dev fp32 [N_pad]; wsum dev int32 [g][N_pad]
+ *            (as produced by rptq_weight_pack and copied to the device); N_pad = ld_w >= N
+ *   bias     NULL or dev fp32 [N_pad]
+ *   act      RPTQ_ACT_NONE or RPTQ_ACT_RELU
+ *   y_dtype  RPTQ_OUT_F32 / RPTQ_OUT_F16: y is dev [M][ldy] of that type (ldy >= N, in elements,
+ *            ldy*sizeof(type) a multiple of 16).
+ *            RPTQ_OUT_CODES: Lout must be given with Lout.K_pad == N; column n of the result is
+ *            padded position n of Lout's layout; y receives M rows of Lout.row_bytes bytes of
+ *            packed codes q' = clamp(rne(v / s'_c') + z'_c'), pad positions 0; ldy is ignored.
+ *   Lout     NULL unless y_dtype == RPTQ_OUT_CODES
+ */
+int rptq_cluster_gemm(const rptq_layout_t* Lin, const void* a_codes, int M, const void* w_codes,
+                      const float* s_w, const int32_t* wsum, int64_t ld_w, const void* bias, int N,
+                      int act, const rptq_layout_t* Lout, void* y, int y_dtype, int64_t ldy,
+                      void* stream);
+
+/*
+ * Raw per-cluster integer accumulators of an output window (Appendix, X~_q,c W~_q,c before
+ * de-quantisation), computed with plain integer instructions and no tensor cores:
+ *   acc[c][m - m0][n - n0] = acc_c[m][n],  m0 <= m < m1 <= M, n0 <= n < n1 <= N
+ * acc is dev int32 [g][m1-m0][n1-n0].
+ */
+int rptq_cluster_gemm_debug_acc(const rptq_layout_t* Lin, const void* a_codes, int M,
+                                const void* w_codes, int N, int m0, int m1, int n0, int n1,
+                                int32_t* acc, void* stream);
+
+/* Host-side readers of the packed formats (format version 1): one byte per code out. */
+int rptq_codes_unpack_host(int K_pad, int bits, const void* packed_host, int64_t M, uint8_t* codes_host);
+int rptq_codes_pack_host(int K_pad, int bits, const uint8_t* codes_host, int64_t M, void* packed_host);
+int rptq_weight_unpack_host(int K_pad, const void* packed_host, int64_t N, int8_t* w_host);
+
+/*
+ * Kernels never spin without a limit: a wait that runs out records RPTQ_ERR_DEVICE_TIMEOUT in a
+ * device status word, lets the block drain and return, and leaves the output undefined. This call
+ * synchronises the device, returns the word in *status (RPTQ_OK if nothing happened) and clears it.
+ */
+int rptq_get_device_status(int* status);
+
+const char* rptq_status_string(int status);
+int rptq_format_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RPTQ_H_ */

@@ -271,27 +271,28 @@ void orc_quantize_clusters(const double* y_r, int64_t M, int C, int g, const int
     free(seg_off);
 }
 
-/* The same quantiser with the decision taken in fp32, the precision the GPU kernel takes it in:
- * t = y * inv_s in one fp32 multiply with inv_s = (float)(1.0 / (double)s), r = rintf(t),
- * q = clamp(r + (float)z, 0, 2^k - 1). Input: fp32 LayerNorm outputs, reordered. With identical
- * inputs the codes must match the GPU's bit for bit. */
+/* The same quantiser with the decision taken from fp32 operands, as the GPU kernel takes it:
+ * Eq. 1's x / s is evaluated as the product of the fp32 value y and the fp32 reciprocal
+ * inv_s = (float)(1.0 / (double)s), and that product is rounded ONCE, half to even, to an integer
+ * (the product of two fp32 numbers is exact in fp64, so nearbyint of the fp64 product is that
+ * single rounding). Then q = clamp(r + z, 0, 2^k - 1). Input: fp32 LayerNorm outputs, reordered.
+ * With identical inputs the codes must match the GPU's bit for bit. */
 void orc_quantize_clusters_f32(const float* y_r, int64_t M, int C, int g, const int32_t* size,
                                const float* scale, const int32_t* zero, int k, int32_t K_pad,
                                uint8_t* codes)
 {
     int32_t* seg_off = (int32_t*)malloc(sizeof(int32_t) * (g + 1));
     orc_segment_offsets(size, g, seg_off);
-    const float qmax = (float)((1 << k) - 1);
+    const double qmax = (double)((1 << k) - 1);
     for (int64_t m = 0; m < M; ++m) {
         uint8_t* row = codes + m * K_pad;
         memset(row, 0, (size_t)K_pad);
         int j = 0;
         for (int c = 0; c < g; ++c) {
-            volatile float inv_s = (float)(1.0 / (double)scale[c]);
+            const float inv_s = (float)(1.0 / (double)scale[c]);
             for (int i = 0; i < size[c]; ++i, ++j) {
-                volatile float t = y_r[m * C + j] * inv_s;
-                float q = rintf(t) + (float)zero[c];
-                if (!(q > 0.0f)) q = 0.0f;
+                double q = nearbyint((double)y_r[m * C + j] * (double)inv_s) + (double)zero[c];
+                if (!(q > 0.0)) q = 0.0;
                 if (q > qmax) q = qmax;
                 row[seg_off[c] + i] = (uint8_t)q;
             }

@@ -1,0 +1,211 @@
+"""Thin Python binding of librptq.so (include/rptq.h): argument marshalling only.
+
+Every step of the hot path runs in the library's CUDA kernels. PyTorch appears here only as the
+owner of device memory and streams. If the library is missing this module raises at import time;
+there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "librptq.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_NOT_BIJECTION, ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_ALLOC = 0, -1, -2, -3, -4, -5, -6
+OUT_F32, OUT_F16, OUT_CODES = 0, 1, 2
+ACT_NONE, ACT_RELU = 0, 1
+
+EXPORTS = (
+    "rptq_layout_create", "rptq_layout_query", "rptq_layout_destroy", "rptq_ln_reorder_quant",
+    "rptq_weight_pack", "rptq_cluster_gemm", "rptq_cluster_gemm_debug_acc", "rptq_codes_unpack_host",
+    "rptq_codes_pack_host", "rptq_weight_unpack_host", "rptq_get_device_status", "rptq_status_string",
+    "rptq_format_version",
+)
+
+
+class RptqError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} ({status})")
+
+
+def _load() -> C.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2304_01089_b200.build` "
+            "(nvcc, sm_100a). There is no CPU or PyTorch fallback.")
+    lib = C.CDLL(LIB_PATH)
+    vp, i32, i64, f32 = C.c_void_p, C.c_int, C.c_int64, C.c_float
+    lib.rptq_layout_create.argtypes = [C.POINTER(vp), i32, i32, i32, vp, vp, vp, vp]
+    lib.rptq_layout_query.argtypes = [vp, C.POINTER(i32), C.POINTER(i64), vp]
+    lib.rptq_layout_destroy.argtypes = [vp]
+    lib.rptq_ln_reorder_quant.argtypes = [vp, vp, i64, vp, vp, f32, i32, vp, vp, vp]
+    lib.rptq_weight_pack.argtypes = [vp, vp, i32, vp, i32, vp, vp, vp]
+    lib.rptq_cluster_gemm.argtypes = [vp, vp, i32, vp, vp, vp, i64, vp, i32, i32, vp, vp, i32, i64, vp]
+    lib.rptq_cluster_gemm_debug_acc.argtypes = [vp, vp, i32, vp, i32, i32, i32, i32, i32, vp, vp]
+    lib.rptq_codes_unpack_host.argtypes = [i32, i32, vp, i64, vp]
+    lib.rptq_codes_pack_host.argtypes = [i32, i32, vp, i64, vp]
+    lib.rptq_weight_unpack_host.argtypes = [i32, vp, i64, vp]
+    lib.rptq_get_device_status.argtypes = [C.POINTER(i32)]
+    lib.rptq_status_string.argtypes = [i32]
+    lib.rptq_status_string.restype = C.c_char_p
+    for name in EXPORTS:
+        if name != "rptq_status_string":
+            getattr(lib, name).restype = i32
+    return lib
+
+
+_lib = _load()
+
+
+def status_string(status: int) -> str:
+    return _lib.rptq_status_string(int(status)).decode()
+
+
+def format_version() -> int:
+    return int(_lib.rptq_format_version())
+
+
+def _check(status: int, where: str) -> None:
+    if status != OK:
+        raise RptqError(status, where)
+
+
+def _np_ptr(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def _dev_ptr(t) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("expected a contiguous CUDA tensor")
+    return t.data_ptr()
+
+
+def _stream_ptr(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+class Layout:
+    """rptq_layout_create / _query / _destroy: reorder index S, cluster sizes, (s_c, z_c)."""
+
+    def __init__(self, perm, cluster_size, scale, zero, bits: int):
+        self._perm = np.ascontiguousarray(perm, dtype=np.int32)
+        self._size = np.ascontiguousarray(cluster_size, dtype=np.int32)
+        self._scale = np.ascontiguousarray(scale, dtype=np.float32)
+        self._zero = np.ascontiguousarray(zero, dtype=np.int32)
+        if not (self._size.shape == self._scale.shape == self._zero.shape):
+            raise ValueError("cluster_size, scale and zero must have one entry per cluster")
+        self.C, self.g, self.bits = int(self._perm.shape[0]), int(self._size.shape[0]), int(bits)
+        h = C.c_void_p()
+        _check(_lib.rptq_layout_create(C.byref(h), self.C, self.g, self.bits, _np_ptr(self._perm),
+                                       _np_ptr(self._size), _np_ptr(self._scale), _np_ptr(self._zero)),
+               "rptq_layout_create")
+        self._h = h
+        k_pad, rb = C.c_int(), C.c_int64()
+        self.seg_off = np.empty(self.g + 1, np.int32)
+        _check(_lib.rptq_layout_query(self._h, C.byref(k_pad), C.byref(rb), _np_ptr(self.seg_off)), "rptq_layout_query")
+        self.K_pad, self.row_bytes = int(k_pad.value), int(rb.value)
+
+    @property
+    def handle(self) -> C.c_void_p:
+        if self._h is None:
+            raise ValueError("layout was destroyed")
+        return self._h
+
+    def destroy(self) -> None:
+        if getattr(self, "_h", None) is not None:
+            _lib.rptq_layout_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+def ln_reorder_quant(layout: Layout, x, gamma, beta, eps: float, codes, y_dbg=None, M: Optional[int] = None,
+                     ldx: Optional[int] = None, stream=None) -> None:
+    """rptq_ln_reorder_quant on device tensors: x fp16 [M][ldx], gamma/beta fp16 [C],
+    codes uint8 [M][row_bytes], y_dbg optional fp32 [M][C]."""
+    M = int(x.shape[0]) if M is None else int(M)
+    ldx = int(x.stride(0)) if ldx is None else int(ldx)
+    _check(_lib.rptq_ln_reorder_quant(layout.handle, _dev_ptr(x), ldx, _dev_ptr(gamma), _dev_ptr(beta),
+                                      C.c_float(eps), M, _dev_ptr(codes), _dev_ptr(y_dbg), _stream_ptr(stream)),
+           "rptq_ln_reorder_quant")
+
+
+def weight_pack(layout_in: Layout, W: np.ndarray, out_perm=None, n_pad: Optional[int] = None):
+    """rptq_weight_pack on host arrays. Returns (w_codes uint8 [N_pad][K_pad/2], s_w fp32 [N_pad],
+    wsum int32 [g][N_pad])."""
+    W = np.ascontiguousarray(W, dtype=np.float32)
+    N, Cn = W.shape
+    if Cn != layout_in.C:
+        raise ValueError("W must be [N][C] with C the layout's channel count")
+    n_pad = N if n_pad is None else int(n_pad)
+    op = None if out_perm is None else np.ascontiguousarray(out_perm, dtype=np.int32)
+    w_codes = np.empty((n_pad, layout_in.K_pad // 2), np.uint8)
+    s_w = np.empty(n_pad, np.float32)
+    wsum = np.empty((layout_in.g, n_pad), np.int32)
+    _check(_lib.rptq_weight_pack(layout_in.handle, _np_ptr(W), N, _np_ptr(op), n_pad, _np_ptr(w_codes),
+                                 _np_ptr(s_w), _np_ptr(wsum)), "rptq_weight_pack")
+    return w_codes, s_w, wsum
+
+
+def cluster_gemm(layout_in: Layout, a_codes, M: int, w_codes, s_w, wsum, N: int, y, *, ld_w: Optional[int] = None,
+                 bias=None, act: int = ACT_NONE, layout_out: Optional[Layout] = None, y_dtype: int = OUT_F32,
+                 ldy: Optional[int] = None, stream=None) -> None:
+    """rptq_cluster_gemm on device tensors."""
+    ld_w = int(s_w.shape[0]) if ld_w is None else int(ld_w)
+    if ldy is None:
+        ldy = 0 if y_dtype == OUT_CODES else int(y.stride(0))
+    _check(_lib.rptq_cluster_gemm(layout_in.handle, _dev_ptr(a_codes), int(M), _dev_ptr(w_codes), _dev_ptr(s_w),
+                                  _dev_ptr(wsum), ld_w, _dev_ptr(bias), int(N), int(act),
+                                  None if layout_out is None else layout_out.handle, _dev_ptr(y), int(y_dtype),
+                                  int(ldy), _stream_ptr(stream)), "rptq_cluster_gemm")
+
+
+def cluster_gemm_debug_acc(layout_in: Layout, a_codes, M: int, w_codes, N: int, m0: int, m1: int, n0: int, n1: int,
+                           acc, stream=None) -> None:
+    _check(_lib.rptq_cluster_gemm_debug_acc(layout_in.handle, _dev_ptr(a_codes), int(M), _dev_ptr(w_codes), int(N),
+                                            int(m0), int(m1), int(n0), int(n1), _dev_ptr(acc), _stream_ptr(stream)),
+           "rptq_cluster_gemm_debug_acc")
+
+
+def codes_unpack_host(packed: np.ndarray, k_pad: int, bits: int) -> np.ndarray:
+    packed = np.ascontiguousarray(packed, dtype=np.uint8)
+    M = packed.shape[0]
+    out = np.empty((M, k_pad), np.uint8)
+    _check(_lib.rptq_codes_unpack_host(int(k_pad), int(bits), _np_ptr(packed), M, _np_ptr(out)), "rptq_codes_unpack_host")
+    return out
+
+
+def codes_pack_host(codes: np.ndarray, bits: int) -> np.ndarray:
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    M, k_pad = codes.shape
+    out = np.empty((M, k_pad * bits // 8), np.uint8)
+    _check(_lib.rptq_codes_pack_host(int(k_pad), int(bits), _np_ptr(codes), M, _np_ptr(out)), "rptq_codes_pack_host")
+    return out
+
+
+def weight_unpack_host(packed: np.ndarray, k_pad: int) -> np.ndarray:
+    packed = np.ascontiguousarray(packed, dtype=np.uint8)
+    N = packed.shape[0]
+    out = np.empty((N, k_pad), np.int8)
+    _check(_lib.rptq_weight_unpack_host(int(k_pad), _np_ptr(packed), N, _np_ptr(out)), "rptq_weight_unpack_host")
+    return out
+
+
+def get_device_status() -> int:
+    s = C.c_int()
+    _check(_lib.rptq_get_device_status(C.byref(s)), "rptq_get_device_status")
+    return int(s.value)

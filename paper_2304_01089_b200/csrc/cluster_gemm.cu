@@ -1,0 +1,594 @@
+// rptq_cluster_gemm: cluster-segmented integer GEMM (Appendix, second computation method).
+//
+//   acc_c[m][n] = sum_{k in segment c} X_q[m][k] * W_q[n][k]        int32, tcgen05.mma kind::i8
+//   y[m][n]     = s_w[n] * sum_c s_c * (acc_c[m][n] - z_c * Wsum_c[n])  (+ bias) (ReLU) (re-quantise)
+//
+// One persistent CTA per SM works on 128 (tokens) x 256 (output channels) tiles. Warp roles:
+//   warp 0      TMA producer: packed activation codes [128 rows x 128 codes] and packed 4-bit
+//               weights [256 rows x 128 codes] per K block into a ring of shared-memory stages
+//   warps 4-7   unpack: packed codes -> 8-bit operands, written in the K-major 128-byte-swizzled
+//               layout that the tensor core reads (weights become 16 * w, see unpack.cuh)
+//   warp 1      MMA issuer: four 128x256x32 tcgen05.mma per K block; each cluster segment
+//               accumulates into one of two 256-column TMEM buffers and is committed when it ends
+//   warps 8-15  epilogue: drain a finished cluster's accumulator (tcgen05.ld), add s_c * acc into
+//               fp32 running sums held in registers while the next cluster's MMAs run; after the
+//               last cluster apply the zero-point correction, s_w, bias, activation, and store
+// Every wait is bounded: a wait that runs out sets RPTQ_ERR_DEVICE_TIMEOUT in the status word and
+// all roles drain and return.
+#include <cuda.h>
+#include <cuda_fp16.h>
+
+#include <mutex>
+
+#include "pack.cuh"
+#include "rptq_internal.h"
+#include "unpack.cuh"
+
+namespace rptq {
+namespace gemm {
+
+constexpr int TILE_M = 128, TILE_N = 256, KBLK = 128;
+constexpr int N_P = 3;            // packed stages
+constexpr int N_U = 2;            // unpacked (operand) stages
+constexpr int THREADS = 512;
+constexpr int UNPACK_WARP0 = 4, N_UNPACK_WARPS = 4;
+constexpr int EPI_WARP0 = 8, N_EPI_WARPS = 8;
+constexpr int A8_BYTES = TILE_M * KBLK, W8_BYTES = TILE_N * KBLK;     // 16 KB, 32 KB
+constexpr int WP_BYTES = TILE_N * KBLK / 2;                           // 16 KB packed weights per stage
+constexpr uint64_t WAIT_BUDGET_NS = 2000000000ull;
+
+__host__ __device__ constexpr int ap_bytes(int bits) { return TILE_M * KBLK * bits / 8; }
+
+struct SmemLayout {
+    int u_stage, p_stage, off_p, off_flags, off_seg_scale, off_cl_sz, off_tab, off_bar, total;
+};
+__host__ __device__ constexpr SmemLayout smem_layout(int bits)
+{
+    SmemLayout s{};
+    s.u_stage = A8_BYTES + W8_BYTES;
+    s.p_stage = ap_bytes(bits) + WP_BYTES;
+    s.off_p = N_U * s.u_stage;
+    s.off_flags = s.off_p + N_P * s.p_stage;
+    s.off_seg_scale = s.off_flags + 2048;
+    s.off_cl_sz = s.off_seg_scale + kMaxGemmSegments * 4;
+    s.off_tab = s.off_cl_sz + kMaxGemmSegments * 4;
+    s.off_bar = s.off_tab + 2 * 3 * TILE_N * 4;
+    s.total = s.off_bar + 256;
+    return s;
+}
+
+struct Params {
+    int M, N, n_kb, n_seg, g;
+    int tiles_m, n_tiles;
+    const uint8_t* step_flags;
+    const float* seg_scale;
+    const float* cl_sz;
+    const float* s_w;
+    const int32_t* wsum;
+    int64_t ld_w;
+    const float* bias;
+    int act, y_dtype;
+    void* y;
+    int64_t ldy;
+    const UnitInfo* out_unit;
+    int out_bits;
+    int64_t out_row_bytes;
+    int* status;
+};
+
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ uint64_t globaltimer_ns()
+{
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait. Returns false when the budget ran out or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, bool heed_abort = true)
+{
+#pragma unroll 1
+    for (int i = 0; i < 128; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = globaltimer_ns();
+#pragma unroll 1
+    while (true) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (heed_abort && *abort_flag) return false;
+        if (globaltimer_ns() - t0 > WAIT_BUDGET_NS) { *abort_flag = 1; return false; }
+    }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_i8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&v)[16])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// K-major operand tile with 128-byte rows and the 128-byte swizzle: 8-row groups are 1024 bytes
+// apart (stride byte offset), the leading byte offset is unused for swizzled K-major layouts.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3FFFFu) >> 4);        // start address, 16-byte units
+    d |= (uint64_t)1 << 16;                         // leading byte offset (ignored)
+    d |= (uint64_t)(1024 >> 4) << 32;               // stride byte offset
+    d |= (uint64_t)1 << 46;                         // descriptor version of this architecture
+    d |= (uint64_t)2 << 61;                         // 128-byte swizzle
+    return d;
+}
+// kind::i8, D = s32, A = unsigned 8-bit (activation codes), B = signed 8-bit (weights), both
+// K-major, M = 128, N = 256.
+constexpr uint32_t kInstrDesc = (2u << 4) | (0u << 7) | (1u << 10) | ((uint32_t)(TILE_N >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
+
+__device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
+{
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ uint32_t lds32(uint32_t addr)
+{
+    uint32_t v;
+    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+    return v;
+}
+
+// One unpack work item: 32 codes of one operand row -> 32 bytes at K offset 32*unit of that row
+// in the swizzled tile (16-byte chunk j of row r lives at chunk position j ^ (r & 7)).
+__device__ __forceinline__ void store_item(uint32_t tile, int row, int unit, const uint32_t (&o)[8])
+{
+    const uint32_t base = tile + row * 128;
+    const int sw = row & 7;
+    sts128(base + (((2 * unit) ^ sw) << 4), o[0], o[1], o[2], o[3]);
+    sts128(base + (((2 * unit + 1) ^ sw) << 4), o[4], o[5], o[6], o[7]);
+}
+
+template <int BITS>
+__global__ void __launch_bounds__(THREADS, 1)
+cluster_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w, const Params p)
+{
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    constexpr SmemLayout SL = smem_layout(BITS);
+    constexpr int AP_BYTES = ap_bytes(BITS);
+    // dynamic shared memory is only guaranteed 16-byte alignment: round up to the swizzle span
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem = smem_raw + (smem_base - smem_u32(smem_raw));
+
+    uint8_t* s_flags = smem + SL.off_flags;
+    float* s_seg_scale = reinterpret_cast<float*>(smem + SL.off_seg_scale);
+    float* s_cl_sz = reinterpret_cast<float*>(smem + SL.off_cl_sz);
+    float* s_tab = reinterpret_cast<float*>(smem + SL.off_tab);           // [2][3][TILE_N]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SL.off_bar);
+    // barrier indices
+    constexpr int B_PFULL = 0, B_PEMPTY = B_PFULL + N_P, B_UFULL = B_PEMPTY + N_P, B_UEMPTY = B_UFULL + N_U,
+                  B_ACCFULL = B_UEMPTY + N_U, B_ACCEMPTY = B_ACCFULL + 2, B_TAB = B_ACCEMPTY + 2, B_DRAIN = B_TAB + 2,
+                  N_BARS = B_DRAIN + 1;
+    static_assert(N_BARS * 8 + 16 <= 256, "barrier block too small");
+    uint32_t* s_tmem_ptr = reinterpret_cast<uint32_t*>(bars + N_BARS);
+    volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem_ptr + 1);
+    const uint32_t bar0 = smem_u32(bars);
+    auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int n_steps = p.n_kb * 4;
+
+    if (tid == 0) {
+        for (int i = 0; i < N_P; ++i) { mbar_init(bar(B_PFULL + i), 1); mbar_init(bar(B_PEMPTY + i), N_UNPACK_WARPS); }
+        for (int i = 0; i < N_U; ++i) { mbar_init(bar(B_UFULL + i), N_UNPACK_WARPS); mbar_init(bar(B_UEMPTY + i), 1); }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(bar(B_ACCFULL + i), 1); mbar_init(bar(B_ACCEMPTY + i), N_EPI_WARPS); mbar_init(bar(B_TAB + i), N_EPI_WARPS);
+        }
+        mbar_init(bar(B_DRAIN), 1);
+        *s_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    for (int i = tid; i < n_steps; i += THREADS) s_flags[i] = p.step_flags[i];
+    for (int i = tid; i < p.n_seg; i += THREADS) s_seg_scale[i] = p.seg_scale[i] * 0.0625f;   // operands were 16 * w
+    for (int i = tid; i < p.g; i += THREADS) s_cl_sz[i] = p.cl_sz[i];
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(s_tmem_ptr)) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *s_tmem_ptr;
+
+
+    // The register file is re-partitioned by warpgroup (the epilogue holds 128 running sums per
+    // thread); each setmaxnreg is executed by the four warps of its group at one place.
+    if (warp < UNPACK_WARP0) {
+      asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
+      if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t n_issued = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < p.n_tiles && ok; t += gridDim.x) {
+                const int m0 = (t % p.tiles_m) * TILE_M, n0 = (t / p.tiles_m) * TILE_N;
+                for (int kb = 0; kb < p.n_kb; ++kb, ++n_issued) {
+                    const int s = n_issued % N_P;
+                    const uint32_t ph = (n_issued / N_P) & 1;
+                    if (!mbar_wait(bar(B_PEMPTY + s), ph ^ 1, s_abort)) { ok = false; break; }
+                    const uint32_t dst = smem_base + SL.off_p + s * SL.p_stage;
+                    mbar_arrive_expect_tx(bar(B_PFULL + s), AP_BYTES + WP_BYTES);
+                    tma_load_2d(dst, &tm_a, kb * (KBLK * BITS / 8), m0, bar(B_PFULL + s));
+                    tma_load_2d(dst + AP_BYTES, &tm_w, kb * (KBLK / 2), n0, bar(B_PFULL + s));
+                }
+            }
+            if (!ok) {
+                // let copies that were already issued land before the CTA's shared memory goes away
+                const uint32_t lo = n_issued > N_P ? n_issued - N_P : 0;
+                for (uint32_t i = lo; i < n_issued; ++i) mbar_wait(bar(B_PFULL + i % N_P), (i / N_P) & 1, s_abort, false);
+            }
+        }
+      } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            uint32_t n_kb_done = 0, n_seg_done = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < p.n_tiles && ok; t += gridDim.x) {
+                for (int kb = 0; kb < p.n_kb && ok; ++kb, ++n_kb_done) {
+                    const int s = n_kb_done % N_U;
+                    if (!mbar_wait(bar(B_UFULL + s), (n_kb_done / N_U) & 1, s_abort)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_tile = smem_base + s * SL.u_stage, w_tile = a_tile + A8_BYTES;
+#pragma unroll 1
+                    for (int j = 0; j < 4; ++j) {
+                        const uint8_t f = s_flags[kb * 4 + j];
+                        if (f & STEP_SKIP) continue;
+                        const uint32_t buf = n_seg_done & 1;
+                        if (f & STEP_FIRST) {
+                            if (!mbar_wait(bar(B_ACCEMPTY + buf), ((n_seg_done >> 1) & 1) ^ 1, s_abort)) { ok = false; break; }
+                            tc_fence_after();
+                        }
+                        tc_mma_i8(tmem_base + buf * TILE_N, smem_desc_sw128(a_tile + j * 32), smem_desc_sw128(w_tile + j * 32),
+                                  kInstrDesc, (f & STEP_FIRST) ? 0u : 1u);
+                        if (f & STEP_LAST) { tc_commit(bar(B_ACCFULL + buf)); ++n_seg_done; }
+                    }
+                    tc_commit(bar(B_UEMPTY + s));      // the stage may be overwritten once these MMAs have read it
+                }
+            }
+            if (!ok) {
+                tc_commit(bar(B_DRAIN));
+                const uint64_t t0 = globaltimer_ns();
+                while (!mbar_try_wait(bar(B_DRAIN), 0) && globaltimer_ns() - t0 < WAIT_BUDGET_NS) {}
+            }
+        }
+      }   // warps 2 and 3 only fill the first warpgroup
+    } else if (warp < EPI_WARP0) {
+        // ------------------------------------------------------------ unpack warps
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");
+        const int ut = tid - UNPACK_WARP0 * 32;      // 0..127
+        uint32_t n_done = 0;
+        bool ok = true;
+        const int total_kb = ((p.n_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x) * p.n_kb;
+        for (int it = 0; it < total_kb; ++it, ++n_done) {
+            const int sp = n_done % N_P, su = n_done % N_U;
+            if (!mbar_wait(bar(B_PFULL + sp), (n_done / N_P) & 1, s_abort)) { ok = false; break; }
+            if (!mbar_wait(bar(B_UEMPTY + su), ((n_done / N_U) & 1) ^ 1, s_abort)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t pa = smem_base + SL.off_p + sp * SL.p_stage, pw = pa + AP_BYTES;
+            const uint32_t a_tile = smem_base + su * SL.u_stage, w_tile = a_tile + A8_BYTES;
+            // activations: 128 rows x 4 units
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int item = ut + i * 128;
+                uint32_t pk[BITS], o[8];
+                if constexpr (BITS == 4) {
+                    const uint4 v = lds128(pa + item * 16);
+                    pk[0] = v.x; pk[1] = v.y; pk[2] = v.z; pk[3] = v.w;
+                } else if constexpr (BITS == 3) {
+#pragma unroll
+                    for (int j = 0; j < 3; ++j) pk[j] = lds32(pa + item * 12 + j * 4);
+                } else {
+                    const uint4 v0 = lds128(pa + item * 32), v1 = lds128(pa + item * 32 + 16);
+                    pk[0] = v0.x; pk[1] = v0.y; pk[2] = v0.z; pk[3] = v0.w;
+                    pk[4] = v1.x; pk[5] = v1.y; pk[6] = v1.z; pk[7] = v1.w;
+                }
+                unpack_act32<BITS>(pk, o);
+                store_item(a_tile, item >> 2, item & 3, o);
+            }
+            // weights: 256 rows x 4 units
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int item = ut + i * 128;
+                const uint4 v = lds128(pw + item * 16);
+                const uint32_t pk[4] = {v.x, v.y, v.z, v.w};
+                uint32_t o[8];
+                unpack_w32_x16(pk, o);
+                store_item(w_tile, item >> 2, item & 3, o);
+            }
+            fence_proxy_async();          // make the generic-proxy stores visible to the tensor core
+            __syncwarp();
+            if (lane == 0) { mbar_arrive(bar(B_UFULL + su)); mbar_arrive(bar(B_PEMPTY + sp)); }
+        }
+        (void)ok;
+    } else {
+        // ------------------------------------------------------------ epilogue warps
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 200;");
+        const int ew = warp - EPI_WARP0;
+        const int q = ew & 3, h = ew >> 2;           // TMEM lane quarter (= warp % 4), column half
+        const int et = ew * 32 + lane;               // 0..255: the column whose tile constants I prepare
+        uint32_t n_seg_done = 0, n_tile_done = 0;
+        bool ok = true;
+        float R[128];
+        for (int t = blockIdx.x; t < p.n_tiles && ok; t += gridDim.x, ++n_tile_done) {
+            const int m0 = (t % p.tiles_m) * TILE_M, n0 = (t / p.tiles_m) * TILE_N;
+            float* tab = s_tab + (n_tile_done & 1) * 3 * TILE_N;
+            {   // per-tile column constants: zero-point correction sum_c s_c z_c Wsum_c[n], s_w[n], bias[n]
+                const int n = n0 + et;
+                float corr = 0.f, sw = 0.f, bs = 0.f;
+                if (n < p.N) {
+                    for (int c = 0; c < p.g; ++c) corr = __fmaf_rn(s_cl_sz[c], (float)__ldg(p.wsum + (int64_t)c * p.ld_w + n), corr);
+                    sw = __ldg(p.s_w + n);
+                    bs = p.bias ? __ldg(p.bias + n) : 0.f;
+                }
+                tab[et] = corr; tab[TILE_N + et] = sw; tab[2 * TILE_N + et] = bs;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(B_TAB + (n_tile_done & 1)));
+            }
+#pragma unroll
+            for (int i = 0; i < 128; ++i) R[i] = 0.f;
+            for (int sgi = 0; sgi < p.n_seg; ++sgi, ++n_seg_done) {
+                const uint32_t buf = n_seg_done & 1;
+                if (!mbar_wait(bar(B_ACCFULL + buf), (n_seg_done >> 1) & 1, s_abort)) { ok = false; break; }
+                tc_fence_after();
+                const float sc = s_seg_scale[sgi];
+                const uint32_t taddr = tmem_base + ((uint32_t)(32 * q) << 16) + buf * TILE_N + h * 128;
+                uint32_t va[16], vb[16];
+                tc_ld16(taddr, va);
+#pragma unroll
+                for (int ch = 0; ch < 8; ch += 2) {
+                    tc_wait_ld();
+                    tc_ld16(taddr + (ch + 1) * 16, vb);
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) R[ch * 16 + i] = __fmaf_rn(sc, (float)(int)va[i], R[ch * 16 + i]);
+                    tc_wait_ld();
+                    if (ch + 2 < 8) tc_ld16(taddr + (ch + 2) * 16, va);
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) R[(ch + 1) * 16 + i] = __fmaf_rn(sc, (float)(int)vb[i], R[(ch + 1) * 16 + i]);
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(B_ACCEMPTY + buf));
+            }
+            if (!ok) break;
+            if (!mbar_wait(bar(B_TAB + (n_tile_done & 1)), (n_tile_done >> 1) & 1, s_abort)) { ok = false; break; }
+            // y = s_w * (R - corr) + bias, activation, store
+            const int m = m0 + 32 * q + lane;
+            const int nb = n0 + h * 128;
+            const float* t_corr = tab + h * 128;
+            const float* t_sw = tab + TILE_N + h * 128;
+            const float* t_bs = tab + 2 * TILE_N + h * 128;
+#pragma unroll
+            for (int i = 0; i < 128; ++i) {
+                float v = __fmaf_rn(t_sw[i], R[i] - t_corr[i], t_bs[i]);
+                if (p.act == RPTQ_ACT_RELU) v = fmaxf(v, 0.f);
+                R[i] = v;
+            }
+            if (m < p.M) {
+                if (p.y_dtype == RPTQ_OUT_F32) {
+                    float* dst = static_cast<float*>(p.y) + (int64_t)m * p.ldy + nb;
+                    if (nb + 128 <= p.N) {
+#pragma unroll
+                        for (int i = 0; i < 128; i += 4) *reinterpret_cast<float4*>(dst + i) = make_float4(R[i], R[i + 1], R[i + 2], R[i + 3]);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 128; ++i) if (nb + i < p.N) dst[i] = R[i];
+                    }
+                } else if (p.y_dtype == RPTQ_OUT_F16) {
+                    __half* dst = static_cast<__half*>(p.y) + (int64_t)m * p.ldy + nb;
+                    if (nb + 128 <= p.N) {
+#pragma unroll
+                        for (int i = 0; i < 128; i += 8) {
+                            __half2 h0 = __floats2half2_rn(R[i], R[i + 1]), h1 = __floats2half2_rn(R[i + 2], R[i + 3]);
+                            __half2 h2 = __floats2half2_rn(R[i + 4], R[i + 5]), h3 = __floats2half2_rn(R[i + 6], R[i + 7]);
+                            uint4 v;
+                            v.x = *reinterpret_cast<uint32_t*>(&h0); v.y = *reinterpret_cast<uint32_t*>(&h1);
+                            v.z = *reinterpret_cast<uint32_t*>(&h2); v.w = *reinterpret_cast<uint32_t*>(&h3);
+                            *reinterpret_cast<uint4*>(dst + i) = v;
+                        }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 128; ++i) if (nb + i < p.N) dst[i] = __float2half_rn(R[i]);
+                    }
+                } else {
+                    // re-quantise for the next site: column n is padded position n of the output layout
+                    uint8_t* row = static_cast<uint8_t*>(p.y) + (int64_t)m * p.out_row_bytes;
+                    const int qmax = (1 << p.out_bits) - 1;
+#pragma unroll
+                    for (int uu = 0; uu < 4; ++uu) {
+                        const int unit = (nb >> 5) + uu;
+                        if (nb + 32 * uu >= p.N) break;
+                        const uint4 t4 = __ldg(reinterpret_cast<const uint4*>(p.out_unit + unit));
+                        const float inv_s = __uint_as_float(t4.x);
+                        const int zc = (int)t4.y, nvalid = (int)t4.w;
+                        uint32_t qv[32];
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) qv[e] = e < nvalid ? quant_code(R[32 * uu + e], inv_s, zc, qmax) : 0u;
+                        if (p.out_bits == 4) {
+                            uint32_t w[4]; pack32<4>(qv, w);
+                            *reinterpret_cast<uint4*>(row + unit * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+                        } else if (p.out_bits == 3) {
+                            uint32_t w[3]; pack32<3>(qv, w);
+                            uint32_t* d = reinterpret_cast<uint32_t*>(row + unit * 12);
+                            d[0] = w[0]; d[1] = w[1]; d[2] = w[2];
+                        } else {
+                            uint32_t w[8]; pack32<8>(qv, w);
+                            uint4* d = reinterpret_cast<uint4*>(row + unit * 32);
+                            d[0] = make_uint4(w[0], w[1], w[2], w[3]); d[1] = make_uint4(w[4], w[5], w[6], w[7]);
+                        }
+                    }
+                }
+            }
+        }
+    }
+
+    // ---------------------------------------------------------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
+    }
+    if (tid == 0 && *s_abort && p.status) atomicExch(p.status, RPTQ_ERR_DEVICE_TIMEOUT);
+}
+
+// ---------------------------------------------------------------- host side
+using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                              const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeFn encode_fn()
+{
+    static std::once_flag once;
+    static EncodeFn fn = nullptr;
+    std::call_once(once, [] {
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeFn>(sym);
+    });
+    return fn;
+}
+
+// 2-D byte tensor [rows][row_bytes], box [box_rows][box_bytes], no swizzle, zero fill out of range.
+static int make_map(CUtensorMap* map, const void* base, uint64_t row_bytes, uint64_t rows, uint32_t box_bytes, uint32_t box_rows)
+{
+    EncodeFn fn = encode_fn();
+    if (!fn) return RPTQ_ERR_CUDA;
+    const cuuint64_t dims[2] = {row_bytes, rows};
+    const cuuint64_t strides[1] = {row_bytes};
+    const cuuint32_t box[2] = {box_bytes, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? RPTQ_OK : RPTQ_ERR_CUDA;
+}
+
+template <int BITS>
+static int launch(const CUtensorMap& tm_a, const CUtensorMap& tm_w, const Params& p, int grid, cudaStream_t st)
+{
+    constexpr SmemLayout SL = smem_layout(BITS);
+    const int smem = SL.total + 1024;     // slack for the in-kernel 1024-byte alignment
+    const void* fn = reinterpret_cast<const void*>(cluster_gemm_kernel<BITS>);
+    cudaFuncAttributes attr;
+    if (cudaFuncGetAttributes(&attr, fn) != cudaSuccess) return RPTQ_ERR_CUDA;
+    // the register re-partition inside the kernel (setmaxnreg) assumes this pool; refuse to launch otherwise
+    if (attr.numRegs * THREADS < 40 * 128 + 64 * 128 + 200 * 256) return RPTQ_ERR_UNSUPPORTED;
+    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return RPTQ_ERR_CUDA;
+    cluster_gemm_kernel<BITS><<<grid, THREADS, smem, st>>>(tm_a, tm_w, p);
+    return cudaGetLastError() == cudaSuccess ? RPTQ_OK : RPTQ_ERR_CUDA;
+}
+
+}  // namespace gemm
+}  // namespace rptq
+
+using namespace rptq;
+
+extern "C" int rptq_cluster_gemm(const rptq_layout_t* Lin, const void* a_codes, int M, const void* w_codes,
+                                 const float* s_w, const int32_t* wsum, int64_t ld_w, const void* bias, int N,
+                                 int act, const rptq_layout_t* Lout, void* y, int y_dtype, int64_t ldy, void* stream)
+{
+    if (!Lin || !a_codes || !w_codes || !s_w || !wsum || !y) return RPTQ_ERR_INVALID_ARG;
+    if (M < 0 || N <= 0 || ld_w < N) return RPTQ_ERR_INVALID_ARG;
+    if (act != RPTQ_ACT_NONE && act != RPTQ_ACT_RELU) return RPTQ_ERR_INVALID_ARG;
+    if (!aligned16(a_codes) || !aligned16(w_codes) || !aligned16(y) || !aligned16(s_w) || !aligned16(wsum) || !aligned16(bias))
+        return RPTQ_ERR_INVALID_ARG;
+    if (y_dtype == RPTQ_OUT_F32) {
+        if (Lout || ldy < N || (ldy * 4) % 16) return RPTQ_ERR_INVALID_ARG;
+    } else if (y_dtype == RPTQ_OUT_F16) {
+        if (Lout || ldy < N || (ldy * 2) % 16) return RPTQ_ERR_INVALID_ARG;
+    } else if (y_dtype == RPTQ_OUT_CODES) {
+        if (!Lout || Lout->K_pad != N) return RPTQ_ERR_INVALID_ARG;
+    } else {
+        return RPTQ_ERR_INVALID_ARG;
+    }
+    if (Lin->g > kMaxGemmSegments || Lin->n_units > 2048) return RPTQ_ERR_UNSUPPORTED;
+    int dev = -1;
+    if (Lin->device < 0 || cudaGetDevice(&dev) != cudaSuccess) return RPTQ_ERR_CUDA;
+    if (dev != Lin->device || (Lout && Lout->device != dev)) return RPTQ_ERR_INVALID_ARG;
+    if (M == 0) return RPTQ_OK;
+
+    gemm::Params p{};
+    p.M = M; p.N = N; p.n_kb = Lin->K_pad / gemm::KBLK; p.n_seg = Lin->n_seg; p.g = Lin->g;
+    p.tiles_m = (M + gemm::TILE_M - 1) / gemm::TILE_M;
+    p.n_tiles = p.tiles_m * ((N + gemm::TILE_N - 1) / gemm::TILE_N);
+    p.step_flags = Lin->d_step_flags; p.seg_scale = Lin->d_seg_scale; p.cl_sz = Lin->d_cl_sz;
+    p.s_w = s_w; p.wsum = wsum; p.ld_w = ld_w; p.bias = static_cast<const float*>(bias);
+    p.act = act; p.y_dtype = y_dtype; p.y = y; p.ldy = ldy;
+    p.out_unit = Lout ? Lout->d_unit : nullptr;
+    p.out_bits = Lout ? Lout->bits : 0;
+    p.out_row_bytes = Lout ? Lout->row_bytes : 0;
+    p.status = device_status_word();
+    if (!p.status) return RPTQ_ERR_ALLOC;
+
+    CUtensorMap tm_a, tm_w;
+    int rc = gemm::make_map(&tm_a, a_codes, (uint64_t)Lin->row_bytes, (uint64_t)M, (uint32_t)(gemm::KBLK * Lin->bits / 8), gemm::TILE_M);
+    if (rc != RPTQ_OK) return rc;
+    rc = gemm::make_map(&tm_w, w_codes, (uint64_t)Lin->K_pad / 2, (uint64_t)ld_w, gemm::KBLK / 2, gemm::TILE_N);
+    if (rc != RPTQ_OK) return rc;
+
+    int n_sm = 0;
+    if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return RPTQ_ERR_CUDA;
+    const int grid = p.n_tiles < n_sm ? p.n_tiles : n_sm;
+    auto st = static_cast<cudaStream_t>(stream);
+    if (Lin->bits == 3) return gemm::launch<3>(tm_a, tm_w, p, grid, st);
+    if (Lin->bits == 4) return gemm::launch<4>(tm_a, tm_w, p, grid, st);
+    return gemm::launch<8>(tm_a, tm_w, p, grid, st);
+}

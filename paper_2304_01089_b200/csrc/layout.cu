@@ -1,0 +1,311 @@
+// Host side of librptq.so: the layout handle (reorder index S with per-cluster parameters,
+// Sec. 4.1), the offline weight preparation (Sec. 4.2), the packed-format readers and the
+// device status word.
+#include <cmath>
+#include <cstring>
+#include <mutex>
+#include <new>
+
+#include "rptq_internal.h"
+
+namespace rptq {
+
+static std::mutex g_status_mutex;
+static int* g_status_word = nullptr;
+
+int* device_status_word()
+{
+    std::lock_guard<std::mutex> lock(g_status_mutex);
+    if (g_status_word == nullptr) {
+        int* p = nullptr;
+        if (cudaMalloc(&p, 256) != cudaSuccess) return nullptr;
+        if (cudaMemset(p, 0, 256) != cudaSuccess) { cudaFree(p); return nullptr; }
+        g_status_word = p;
+    }
+    return g_status_word;
+}
+
+template <class T>
+static int upload(T** dst, const T* src, size_t n)
+{
+    if (n == 0) n = 1;
+    if (cudaMalloc(reinterpret_cast<void**>(dst), n * sizeof(T)) != cudaSuccess) return RPTQ_ERR_ALLOC;
+    if (src && cudaMemcpy(*dst, src, n * sizeof(T), cudaMemcpyHostToDevice) != cudaSuccess) return RPTQ_ERR_CUDA;
+    return RPTQ_OK;
+}
+
+// ---- packed formats, word at a time ------------------------------------------------------------
+// 4-bit: word = lo | hi << 4 where lo holds codes 0..3 one per byte and hi codes 4..7.
+static inline uint32_t word_of_bytes(const uint8_t* c) { return c[0] | (c[1] << 8) | (c[2] << 16) | ((uint32_t)c[3] << 24); }
+
+static void pack_row(const uint8_t* codes, int K_pad, int bits, uint8_t* out)
+{
+    if (bits == 8) { std::memcpy(out, codes, (size_t)K_pad); return; }
+    uint32_t* w = reinterpret_cast<uint32_t*>(out);
+    if (bits == 4) {
+        for (int i = 0; i < K_pad / 8; ++i)
+            w[i] = (word_of_bytes(codes + 8 * i) & 0x0F0F0F0Fu) | ((word_of_bytes(codes + 8 * i + 4) & 0x0F0F0F0Fu) << 4);
+        return;
+    }
+    for (int grp = 0; grp < K_pad / 32; ++grp) {
+        const uint8_t* c = codes + 32 * grp;
+        uint32_t tail = (word_of_bytes(c + 24) & 0x07070707u) | ((word_of_bytes(c + 28) & 0x07070707u) << 4);
+        for (int j = 0; j < 3; ++j) {
+            uint32_t body = (word_of_bytes(c + 8 * j) & 0x07070707u) | ((word_of_bytes(c + 8 * j + 4) & 0x07070707u) << 4);
+            w[3 * grp + j] = body | (((tail >> j) & 0x11111111u) << 3);
+        }
+    }
+}
+
+static inline void bytes_of_word(uint32_t v, uint8_t* c) { c[0] = v; c[1] = v >> 8; c[2] = v >> 16; c[3] = v >> 24; }
+
+static void unpack_row(const uint8_t* in, int K_pad, int bits, uint8_t* codes)
+{
+    if (bits == 8) { std::memcpy(codes, in, (size_t)K_pad); return; }
+    const uint32_t* w = reinterpret_cast<const uint32_t*>(in);
+    if (bits == 4) {
+        for (int i = 0; i < K_pad / 8; ++i) {
+            bytes_of_word(w[i] & 0x0F0F0F0Fu, codes + 8 * i);
+            bytes_of_word((w[i] >> 4) & 0x0F0F0F0Fu, codes + 8 * i + 4);
+        }
+        return;
+    }
+    for (int grp = 0; grp < K_pad / 32; ++grp) {
+        uint32_t tail = 0;
+        for (int j = 0; j < 3; ++j) {
+            uint32_t v = w[3 * grp + j];
+            bytes_of_word(v & 0x07070707u, codes + 32 * grp + 8 * j);
+            bytes_of_word((v >> 4) & 0x07070707u, codes + 32 * grp + 8 * j + 4);
+            tail |= ((v >> 3) & 0x11111111u) << j;
+        }
+        bytes_of_word(tail & 0x07070707u, codes + 32 * grp + 24);
+        bytes_of_word((tail >> 4) & 0x07070707u, codes + 32 * grp + 28);
+    }
+}
+
+}  // namespace rptq
+
+using namespace rptq;
+
+extern "C" {
+
+int rptq_format_version(void) { return RPTQ_FORMAT_VERSION; }
+
+const char* rptq_status_string(int status)
+{
+    switch (status) {
+        case RPTQ_OK: return "ok";
+        case RPTQ_ERR_INVALID_ARG: return "invalid argument";
+        case RPTQ_ERR_UNSUPPORTED: return "unsupported size or option";
+        case RPTQ_ERR_NOT_BIJECTION: return "reorder index is not a bijection";
+        case RPTQ_ERR_CUDA: return "CUDA call failed";
+        case RPTQ_ERR_DEVICE_TIMEOUT: return "bounded wait inside a kernel ran out";
+        case RPTQ_ERR_ALLOC: return "allocation failed";
+        default: return "unknown status";
+    }
+}
+
+int rptq_get_device_status(int* status)
+{
+    if (!status) return RPTQ_ERR_INVALID_ARG;
+    int* word = device_status_word();
+    if (!word) return RPTQ_ERR_ALLOC;
+    if (cudaDeviceSynchronize() != cudaSuccess) return RPTQ_ERR_CUDA;
+    int v = 0;
+    if (cudaMemcpy(&v, word, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return RPTQ_ERR_CUDA;
+    if (v != 0 && cudaMemset(word, 0, sizeof(int)) != cudaSuccess) return RPTQ_ERR_CUDA;
+    *status = v;
+    return RPTQ_OK;
+}
+
+int rptq_layout_create(rptq_layout_t** out, int C, int g, int bits, const int32_t* perm_host,
+                       const int32_t* cluster_size, const float* scale_host, const int32_t* zero_host)
+{
+    if (!out) return RPTQ_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!perm_host || !cluster_size || !scale_host || !zero_host) return RPTQ_ERR_INVALID_ARG;
+    if (C <= 0 || g <= 0) return RPTQ_ERR_INVALID_ARG;
+    if (bits != 3 && bits != 4 && bits != 8) return RPTQ_ERR_UNSUPPORTED;
+    if (C % 8 != 0 || C < 8 || C > 65528 || g > 4096) return RPTQ_ERR_UNSUPPORTED;
+
+    // S must be a bijection and the sizes must tile it
+    std::vector<uint8_t> seen((size_t)C, 0);
+    for (int j = 0; j < C; ++j) {
+        int32_t c = perm_host[j];
+        if (c < 0 || c >= C || seen[c]) return RPTQ_ERR_NOT_BIJECTION;
+        seen[c] = 1;
+    }
+    int64_t total = 0, padded = 0;
+    for (int c = 0; c < g; ++c) {
+        if (cluster_size[c] < 0) return RPTQ_ERR_INVALID_ARG;
+        total += cluster_size[c];
+        padded += (cluster_size[c] + 31) / 32 * 32;
+        if (!(scale_host[c] > 0.0f) || !std::isfinite(scale_host[c])) return RPTQ_ERR_INVALID_ARG;
+        if (zero_host[c] <= -(1 << 21) || zero_host[c] >= (1 << 21)) return RPTQ_ERR_UNSUPPORTED;
+    }
+    if (total != C) return RPTQ_ERR_NOT_BIJECTION;
+    int64_t k_pad = (padded + 127) / 128 * 128;
+    if (k_pad < 128) k_pad = 128;
+    if (k_pad > 65408) return RPTQ_ERR_UNSUPPORTED;
+
+    rptq_layout* L = new (std::nothrow) rptq_layout();
+    if (!L) return RPTQ_ERR_ALLOC;
+    L->C = C; L->g = g; L->bits = bits; L->K_pad = (int)k_pad;
+    L->row_bytes = k_pad * bits / 8;
+    L->n_units = (int)(k_pad / 32);
+    L->perm.assign(perm_host, perm_host + C);
+    L->size.assign(cluster_size, cluster_size + g);
+    L->scale.assign(scale_host, scale_host + g);
+    L->zero.assign(zero_host, zero_host + g);
+    L->seg_off.resize((size_t)g + 1);
+    // Without a CUDA device the handle is host-only: rptq_weight_pack and rptq_layout_query work,
+    // kernel launches report RPTQ_ERR_CUDA.
+    int n_dev = 0;
+    const bool have_device = cudaGetDeviceCount(&n_dev) == cudaSuccess && n_dev > 0;
+    if (!have_device) (void)cudaGetLastError();
+    if (have_device && cudaGetDevice(&L->device) != cudaSuccess) { delete L; return RPTQ_ERR_CUDA; }
+
+    std::vector<uint16_t> src((size_t)k_pad, (uint16_t)C);
+    std::vector<UnitInfo> unit((size_t)L->n_units);
+    std::vector<uint8_t> flags((size_t)L->n_units, STEP_SKIP);
+    std::vector<float> seg_scale, cl_sz((size_t)g);
+    for (auto& u : unit) { u.inv_s = 1.0f; u.zc = 0 - 0x4B400000; u.j0 = 0; u.nvalid = 0; }
+    int off = 0, j = 0;
+    for (int c = 0; c < g; ++c) {
+        L->seg_off[c] = off;
+        const int n = cluster_size[c];
+        const float inv_s = (float)(1.0 / (double)scale_host[c]);
+        cl_sz[c] = scale_host[c] * (float)zero_host[c];
+        const int units_here = (n + 31) / 32;
+        for (int u = 0; u < units_here; ++u) {
+            UnitInfo& ui = unit[off / 32 + u];
+            ui.inv_s = inv_s;
+            ui.zc = zero_host[c] - 0x4B400000;
+            ui.j0 = j + 32 * u;
+            ui.nvalid = (n - 32 * u) < 32 ? (n - 32 * u) : 32;
+            flags[off / 32 + u] = (u == 0 ? STEP_FIRST : 0) | (u == units_here - 1 ? STEP_LAST : 0);
+        }
+        for (int i = 0; i < n; ++i) src[off + i] = (uint16_t)ybuf_addr(perm_host[j + i], C);
+        if (n > 0) { seg_scale.push_back(scale_host[c]); L->n_seg++; }
+        j += n;
+        off += units_here * 32;
+    }
+    L->seg_off[g] = off;
+
+    if (!have_device) { *out = L; return RPTQ_OK; }
+    int rc = upload(&L->d_src, src.data(), src.size());
+    if (rc == RPTQ_OK) rc = upload(&L->d_unit, unit.data(), unit.size());
+    if (rc == RPTQ_OK) rc = upload(&L->d_step_flags, flags.data(), flags.size());
+    if (rc == RPTQ_OK) rc = upload(&L->d_seg_scale, seg_scale.data(), seg_scale.size());
+    if (rc == RPTQ_OK) rc = upload(&L->d_cl_sz, cl_sz.data(), cl_sz.size());
+    if (rc == RPTQ_OK) rc = upload(&L->d_seg_off, L->seg_off.data(), L->seg_off.size());
+    if (rc != RPTQ_OK) { rptq_layout_destroy(L); return rc; }
+    *out = L;
+    return RPTQ_OK;
+}
+
+int rptq_layout_query(const rptq_layout_t* L, int* K_pad, int64_t* row_bytes, int32_t* seg_offset_out)
+{
+    if (!L) return RPTQ_ERR_INVALID_ARG;
+    if (K_pad) *K_pad = L->K_pad;
+    if (row_bytes) *row_bytes = L->row_bytes;
+    if (seg_offset_out) std::memcpy(seg_offset_out, L->seg_off.data(), sizeof(int32_t) * ((size_t)L->g + 1));
+    return RPTQ_OK;
+}
+
+int rptq_layout_destroy(rptq_layout_t* L)
+{
+    if (!L) return RPTQ_OK;
+    cudaFree(L->d_src);
+    cudaFree(L->d_unit);
+    cudaFree(L->d_step_flags);
+    cudaFree(L->d_seg_scale);
+    cudaFree(L->d_cl_sz);
+    cudaFree(L->d_seg_off);
+    delete L;
+    return RPTQ_OK;
+}
+
+int rptq_codes_pack_host(int K_pad, int bits, const uint8_t* codes_host, int64_t M, void* packed_host)
+{
+    if (!codes_host || !packed_host || M < 0 || K_pad <= 0 || K_pad % 128) return RPTQ_ERR_INVALID_ARG;
+    if (bits != 3 && bits != 4 && bits != 8) return RPTQ_ERR_UNSUPPORTED;
+    const int64_t rb = (int64_t)K_pad * bits / 8;
+    for (int64_t m = 0; m < M; ++m) pack_row(codes_host + m * K_pad, K_pad, bits, static_cast<uint8_t*>(packed_host) + m * rb);
+    return RPTQ_OK;
+}
+
+int rptq_codes_unpack_host(int K_pad, int bits, const void* packed_host, int64_t M, uint8_t* codes_host)
+{
+    if (!codes_host || !packed_host || M < 0 || K_pad <= 0 || K_pad % 128) return RPTQ_ERR_INVALID_ARG;
+    if (bits != 3 && bits != 4 && bits != 8) return RPTQ_ERR_UNSUPPORTED;
+    const int64_t rb = (int64_t)K_pad * bits / 8;
+    for (int64_t m = 0; m < M; ++m) unpack_row(static_cast<const uint8_t*>(packed_host) + m * rb, K_pad, bits, codes_host + m * K_pad);
+    return RPTQ_OK;
+}
+
+int rptq_weight_unpack_host(int K_pad, const void* packed_host, int64_t N, int8_t* w_host)
+{
+    if (!w_host || !packed_host || N < 0 || K_pad <= 0 || K_pad % 128) return RPTQ_ERR_INVALID_ARG;
+    const int64_t rb = K_pad / 2;
+    for (int64_t n = 0; n < N; ++n) {
+        uint8_t* dst = reinterpret_cast<uint8_t*>(w_host) + n * K_pad;
+        unpack_row(static_cast<const uint8_t*>(packed_host) + n * rb, K_pad, 4, dst);
+        for (int p = 0; p < K_pad; ++p) dst[p] = (uint8_t)((dst[p] ^ 8u) - 8u);   // sign-extend the nibble
+    }
+    return RPTQ_OK;
+}
+
+int rptq_weight_pack(const rptq_layout_t* Lin, const float* W_host, int N, const int32_t* out_perm,
+                     int N_pad, void* w_codes_host, float* s_w, int32_t* wsum)
+{
+    if (!Lin || !W_host || !w_codes_host || !s_w || !wsum) return RPTQ_ERR_INVALID_ARG;
+    if (N <= 0 || N_pad < N) return RPTQ_ERR_INVALID_ARG;
+    const int C = Lin->C, g = Lin->g, K_pad = Lin->K_pad;
+    if (out_perm) {
+        std::vector<uint8_t> seen((size_t)N, 0);
+        for (int r = 0; r < N; ++r) {
+            if (out_perm[r] < 0 || out_perm[r] >= N || seen[out_perm[r]]) return RPTQ_ERR_NOT_BIJECTION;
+            seen[out_perm[r]] = 1;
+        }
+    }
+    const int64_t rb = K_pad / 2;
+    uint8_t* packed = static_cast<uint8_t*>(w_codes_host);
+    int failed = 0;
+#pragma omp parallel
+    {
+        std::vector<uint8_t> row((size_t)K_pad);
+#pragma omp for schedule(static)
+        for (int r = 0; r < N_pad; ++r) {
+            std::memset(row.data(), 0, (size_t)K_pad);
+            float s = 1.0f;
+            if (r < N) {
+                const float* w = W_host + (int64_t)(out_perm ? out_perm[r] : r) * C;
+                float amax = 0.0f;
+                for (int k = 0; k < C; ++k) amax = fmaxf(amax, fabsf(w[k]));
+                if (!std::isfinite(amax)) failed = 1;
+                if (amax > 0.0f) s = amax / 7.0f;
+                int j = 0;
+                for (int c = 0; c < g; ++c) {
+                    int32_t sum = 0;
+                    uint8_t* seg = row.data() + Lin->seg_off[c];
+                    for (int i = 0; i < Lin->size[c]; ++i, ++j) {
+                        float q = rintf(w[Lin->perm[j]] / s);
+                        q = fminf(fmaxf(q, -8.0f), 7.0f);
+                        const int qi = (int)q;
+                        sum += qi;
+                        seg[i] = (uint8_t)(qi & 0xF);
+                    }
+                    wsum[(int64_t)c * N_pad + r] = sum;
+                }
+            } else {
+                for (int c = 0; c < g; ++c) wsum[(int64_t)c * N_pad + r] = 0;
+            }
+            s_w[r] = s;
+            pack_row(row.data(), K_pad, 4, packed + r * rb);
+        }
+    }
+    return failed ? RPTQ_ERR_INVALID_ARG : RPTQ_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,43 @@
+// Device-side writer of the packed code formats (format version 1, described in rptq.h):
+// 32 consecutive codes, one per register, become BITS 32-bit words.
+#pragma once
+#include <stdint.h>
+
+namespace rptq {
+
+// The quantiser decision shared by both kernels: t = y * inv_s rounded ONCE to an integer, half to
+// even (the fused multiply-add forms the product exactly; adding 1.5 * 2^23 leaves the rounded
+// integer in the low mantissa bits for |t| < 2^22 and keeps order beyond), then + z_c and clamp.
+// zc = z_c - 0x4B400000 (the bit pattern of 1.5 * 2^23).
+__device__ __forceinline__ uint32_t quant_code(float y, float inv_s, int zc, int qmax)
+{
+    const float v = __fmaf_rn(y, inv_s, 12582912.0f);
+    const int q = __float_as_int(v) + zc;
+    return (uint32_t)min(max(q, 0), qmax);
+}
+
+__device__ __forceinline__ uint32_t nibble_word(const uint32_t* q)   // 8 codes -> one 4-bit-layout word
+{
+    uint32_t w = 0;
+#pragma unroll
+    for (int t = 0; t < 8; ++t) w |= q[t] << (8 * (t & 3) + 4 * (t >> 2));
+    return w;
+}
+
+template <int BITS>
+__device__ __forceinline__ void pack32(const uint32_t (&q)[32], uint32_t (&w)[BITS])
+{
+    if constexpr (BITS == 8) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) w[i] = q[4 * i] | (q[4 * i + 1] << 8) | (q[4 * i + 2] << 16) | (q[4 * i + 3] << 24);
+    } else if constexpr (BITS == 4) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) w[i] = nibble_word(q + 8 * i);
+    } else {
+        const uint32_t tail = nibble_word(q + 24);
+#pragma unroll
+        for (int j = 0; j < 3; ++j) w[j] = nibble_word(q + 8 * j) | (((tail >> j) & 0x11111111u) << 3);
+    }
+}
+
+}  // namespace rptq

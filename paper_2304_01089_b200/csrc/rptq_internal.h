@@ -1,0 +1,57 @@
+// Internal declarations shared by the translation units of librptq.so. Not part of the C boundary.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "rptq.h"
+
+namespace rptq {
+
+// One entry per group of 32 padded positions ("unit"). A unit never straddles two clusters
+// because every cluster segment starts at a multiple of 32.
+struct UnitInfo {
+    float inv_s;      // (float)(1.0 / (double)s_c)
+    int32_t zc;       // z_c - 0x4B400000: added to the bit pattern of (t + 1.5*2^23)
+    int32_t j0;       // reordered channel index of the unit's first position
+    int32_t nvalid;   // real (non-pad) positions in the unit, 0..32; real ones come first
+};
+static_assert(sizeof(UnitInfo) == 16, "UnitInfo is loaded as one 16-byte vector");
+
+// Flags of one contraction step (32 consecutive padded positions) along K.
+enum : uint8_t { STEP_FIRST = 1, STEP_LAST = 2, STEP_SKIP = 4 };
+
+constexpr int kMaxGemmSegments = 1024;
+
+// Shared-memory slot (in floats) of channel c of a normalised row in rptq_ln_reorder_quant. The
+// two 16-byte halves of each 8-channel chunk live in separate regions so that both vector stores
+// of a warp are contiguous across lanes; slot C holds the value that pad positions read.
+__host__ __device__ inline int ybuf_addr(int c, int C) { return ((c >> 3) << 2) + (c & 3) + ((c >> 2) & 1) * (C >> 1); }
+
+}  // namespace rptq
+
+struct rptq_layout {
+    int C = 0, g = 0, bits = 0, K_pad = 0, device = -1;
+    int64_t row_bytes = 0;
+    int n_units = 0;   // K_pad / 32
+    int n_seg = 0;     // clusters with n_c > 0
+    std::vector<int32_t> perm, size, seg_off, zero;
+    std::vector<float> scale;
+    // device tables
+    uint16_t* d_src = nullptr;          // [K_pad] ybuf_addr of each padded position's channel, C = pad
+    rptq::UnitInfo* d_unit = nullptr;   // [n_units]
+    uint8_t* d_step_flags = nullptr;    // [n_units]
+    float* d_seg_scale = nullptr;       // [n_seg]  s_c of the non-empty clusters, in K order
+    float* d_cl_sz = nullptr;           // [g]      s_c * z_c
+    int32_t* d_seg_off = nullptr;       // [g+1]    padded segment offsets
+};
+
+namespace rptq {
+
+int* device_status_word();   // lazily allocated device int, RPTQ_OK when clear; nullptr on failure
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace rptq

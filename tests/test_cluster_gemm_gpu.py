@@ -1,0 +1,241 @@
+"""Parity of rptq_cluster_gemm (tcgen05 path, through the C boundary) against the CPU oracle.
+
+Inputs of the GEMM (packed activation codes, packed weights, s_w, Wsum) are produced by the
+oracle here, so a fault in rptq_ln_reorder_quant or rptq_weight_pack cannot hide one in the GEMM.
+"""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2304_01089_b200 import workloads
+from helpers import Site, random_layout_params
+
+pytestmark = pytest.mark.gpu
+
+TOL = 1e-4   # max |dy| <= TOL * max |y| on the fp32 output
+
+
+def _case(rng, M, N, C, g, bits, n_pad=None, allow_empty=True):
+    perm, size, scale, zero = random_layout_params(rng, C, g, bits, allow_empty)
+    n_pad = N if n_pad is None else n_pad
+    W = (rng.normal(size=(N, C)) * 0.02).astype(np.float32)
+    w_codes, s_w, wsum = oracle.weight_quantize(W, perm, size, None, n_pad)
+    off, k_pad = oracle.segment_offsets(size)
+    a = np.zeros((M, k_pad), np.uint8)
+    for c in range(g):
+        a[:, off[c]:off[c] + size[c]] = rng.integers(0, 1 << bits, size=(M, size[c]))
+    return dict(perm=perm, size=size, scale=scale, zero=zero, w_codes=w_codes, s_w=s_w, wsum=wsum,
+                a=a, k_pad=k_pad, bits=bits, M=M, N=N, n_pad=n_pad)
+
+
+def _dev(case):
+    import torch
+    from paper_2304_01089_b200 import binding
+    L = binding.Layout(case["perm"], case["size"], case["scale"], case["zero"], case["bits"])
+    assert L.K_pad == case["k_pad"]
+    d = dict(L=L,
+             a=torch.from_numpy(oracle.pack(case["a"], case["bits"])).cuda(),
+             w=torch.from_numpy(oracle.pack_weights(case["w_codes"])).cuda(),
+             s_w=torch.from_numpy(case["s_w"]).cuda(),
+             wsum=torch.from_numpy(case["wsum"]).cuda())
+    return d
+
+
+def _gemm(case, d, y_dtype=0, bias=None, act=0, layout_out=None, ldy=None, s_w=None, wsum=None, L=None):
+    import torch
+    from paper_2304_01089_b200 import binding
+    M, N = case["M"], case["N"]
+    L = d["L"] if L is None else L
+    if y_dtype == binding.OUT_CODES:
+        y = torch.full((M + 1, layout_out.row_bytes), 0xA5, dtype=torch.uint8, device="cuda")
+    else:
+        ldy = N if ldy is None else ldy
+        dt = torch.float32 if y_dtype == binding.OUT_F32 else torch.float16
+        y = torch.full((M + 1, ldy), float("nan"), dtype=dt, device="cuda")
+    bd = None if bias is None else torch.from_numpy(bias).cuda()
+    binding.cluster_gemm(L, d["a"], M, d["w"], d["s_w"] if s_w is None else s_w, d["wsum"] if wsum is None else wsum,
+                         N, y, ld_w=case["n_pad"], bias=bd, act=act, layout_out=layout_out, y_dtype=y_dtype,
+                         ldy=None if y_dtype == binding.OUT_CODES else y.stride(0))
+    torch.cuda.synchronize()
+    assert binding.get_device_status() == 0
+    out = y.cpu().numpy()
+    if y_dtype == binding.OUT_CODES:
+        assert np.all(out[M] == 0xA5)
+    else:
+        assert np.all(np.isnan(out[M].astype(np.float32))), "wrote past the last row"
+        if out.shape[1] > N:
+            assert np.all(np.isnan(out[:M, N:].astype(np.float32))), "wrote past the last column"
+    return out[:M]
+
+
+def _oracle_y(case, bias=None, relu=False, rows=None):
+    a = case["a"] if rows is None else case["a"][rows]
+    return oracle.cluster_gemm(a, case["w_codes"][:case["N"]], case["size"], case["scale"].astype(np.float64),
+                               case["zero"], case["s_w"], case["wsum"], bias=bias, relu=relu)
+
+
+@pytest.mark.parametrize("bits", [4, 3, 8])
+def test_per_cluster_accumulators_are_bit_exact(bits):
+    """Each cluster's integer accumulator, read out through the epilogue by giving that cluster
+    scale 1 and every other cluster a vanishing scale, with s_w = 1 and z = 0; and the same
+    accumulators from the integer-instruction debug kernel."""
+    import torch
+    from paper_2304_01089_b200 import binding
+    rng = np.random.default_rng(bits)
+    case = _case(rng, M=200, N=300, C=448, g=4, bits=bits, n_pad=304)
+    d = _dev(case)
+    want = oracle.cluster_acc(case["a"], case["w_codes"][:case["N"]], case["size"])
+    ones = torch.ones(case["n_pad"], dtype=torch.float32, device="cuda")
+    zeros_ws = torch.zeros_like(d["wsum"])
+    for c in range(4):
+        if case["size"][c] == 0:
+            continue
+        scale = np.full(4, 2.0 ** -80, np.float32)
+        scale[c] = 1.0
+        L = binding.Layout(case["perm"], case["size"], scale, np.zeros(4, np.int32), bits)
+        y = _gemm(case, d, s_w=ones, wsum=zeros_ws, L=L, ldy=304)[:, :case["N"]]
+        assert np.array_equal(y.astype(np.int64), want[c]), f"cluster {c}"
+    acc = torch.full((4, 200, 300), -1, dtype=torch.int32, device="cuda")
+    binding.cluster_gemm_debug_acc(d["L"], d["a"], 200, d["w"], 300, 0, 200, 0, 300, acc)
+    torch.cuda.synchronize()
+    assert np.array_equal(acc.cpu().numpy().astype(np.int64), want)
+    win = torch.full((4, 7, 9), -1, dtype=torch.int32, device="cuda")
+    binding.cluster_gemm_debug_acc(d["L"], d["a"], 200, d["w"], 300, 100, 107, 250, 259, win)
+    torch.cuda.synchronize()
+    assert np.array_equal(win.cpu().numpy().astype(np.int64), want[:, 100:107, 250:259])
+
+
+@pytest.mark.parametrize("bits", [4, 3, 8])
+@pytest.mark.parametrize("M,N,C,g", [(1, 256, 128, 1), (127, 200, 384, 5), (129, 520, 640, 7), (300, 256, 1024, 33)])
+def test_small_and_ragged_shapes(bits, M, N, C, g):
+    from paper_2304_01089_b200 import binding
+    rng = np.random.default_rng(1000 * bits + M + N)
+    n_pad = (N + 7) // 8 * 8
+    case = _case(rng, M, N, C, g, bits, n_pad=n_pad)
+    d = _dev(case)
+    want = _oracle_y(case)
+    y32 = _gemm(case, d, ldy=n_pad + 8)[:, :N]
+    assert np.max(np.abs(y32 - want)) <= TOL * np.abs(want).max()
+    # fp16 output: the same fp32 result rounded once to fp16
+    y16 = _gemm(case, d, y_dtype=binding.OUT_F16, ldy=n_pad + 8)[:, :N]
+    assert np.array_equal(y16, y32.astype(np.float16))
+    # bias and ReLU
+    bias = (rng.normal(size=n_pad) * np.abs(want).mean()).astype(np.float32)
+    yb = _gemm(case, d, bias=bias, act=binding.ACT_RELU, ldy=n_pad + 8)[:, :N]
+    want_b = _oracle_y(case, bias=bias[:N], relu=True)
+    assert np.max(np.abs(yb - want_b)) <= TOL * np.abs(want).max()
+    assert yb.min() >= 0.0
+
+
+def test_two_launches_on_two_streams_give_identical_bytes():
+    import torch
+    from paper_2304_01089_b200 import binding
+    rng = np.random.default_rng(77)
+    case = _case(rng, 513, 768, 1536, 9, 4)
+    d = _dev(case)
+    y1 = _gemm(case, d)
+    s2 = torch.cuda.Stream()
+    y = torch.empty((513, 768), dtype=torch.float32, device="cuda")
+    binding.cluster_gemm(d["L"], d["a"], 513, d["w"], d["s_w"], d["wsum"], 768, y, stream=s2)
+    torch.cuda.synchronize()
+    assert np.array_equal(y.cpu().numpy(), y1)
+
+
+@pytest.mark.parametrize("out_bits", [4, 3, 8])
+def test_requantised_output_feeds_the_next_layer(out_bits):
+    """FC1 -> ReLU -> quantise in the next site's cluster order -> FC2 (Sec. 4.2: FC1's rows follow
+    the next reorder index; FC2's output keeps the original channel order)."""
+    import torch
+    from paper_2304_01089_b200 import binding
+    rng = np.random.default_rng(40 + out_bits)
+    M, C, H, g1, g2 = 150, 256, 800, 4, 6          # hidden width H is the second site's channel count
+    perm1, size1, scale1, zero1 = random_layout_params(rng, C, g1, 4)
+    perm2, size2, _, _ = random_layout_params(rng, H, g2, out_bits)
+    off2, k_pad2 = oracle.segment_offsets(size2)
+    # FC1's output rows in the second site's padded order: row r = original hidden channel or a zero pad
+    out_rows = np.full(k_pad2, -1, np.int64)
+    j = 0
+    for c in range(g2):
+        out_rows[off2[c]:off2[c] + size2[c]] = perm2[j:j + size2[c]]
+        j += size2[c]
+    W1 = (rng.normal(size=(H, C)) * 0.02).astype(np.float32)
+    W1p = np.zeros((k_pad2, C), np.float32)
+    W1p[out_rows >= 0] = W1[out_rows[out_rows >= 0]]
+    b1 = np.zeros(k_pad2, np.float32)
+    b1[out_rows >= 0] = (rng.normal(size=H) * 0.05).astype(np.float32)[out_rows[out_rows >= 0]]
+    w1_codes, s_w1, wsum1 = oracle.weight_quantize(W1p, perm1, size1, None, k_pad2)
+    off1, k_pad1 = oracle.segment_offsets(size1)
+    a = np.zeros((M, k_pad1), np.uint8)
+    for c in range(g1):
+        a[:, off1[c]:off1[c] + size1[c]] = rng.integers(0, 16, size=(M, size1[c]))
+    case1 = dict(perm=perm1, size=size1, scale=scale1, zero=zero1, w_codes=w1_codes, s_w=s_w1, wsum=wsum1, a=a,
+                 k_pad=k_pad1, bits=4, M=M, N=k_pad2, n_pad=k_pad2)
+    d1 = _dev(case1)
+    h64 = _oracle_y(case1, bias=b1, relu=True)                     # [M][k_pad2], padded order
+    real = out_rows >= 0
+    # second-site parameters from the observed range of h (Eq. 2 per cluster)
+    scale2, zero2 = np.ones(g2, np.float32), np.zeros(g2, np.int32)
+    for c in range(g2):
+        if size2[c]:
+            seg = h64[:, off2[c]:off2[c] + size2[c]]
+            s, z = oracle.minmax_params(seg.min(), seg.max(), out_bits)
+            scale2[c], zero2[c] = s, z
+    L2 = binding.Layout(perm2, size2, scale2, zero2, out_bits)
+    assert L2.K_pad == k_pad2
+    # GPU: fp32 output and re-quantised output of the same launch parameters
+    h32 = _gemm(case1, d1, bias=b1, act=binding.ACT_RELU)
+    packed = _gemm(case1, d1, y_dtype=binding.OUT_CODES, bias=b1, act=binding.ACT_RELU, layout_out=L2)
+    got = oracle.unpack(packed, k_pad2, out_bits)
+    # the decision, bit for bit, from the GPU's own fp32 values (real positions in reordered order)
+    want32 = oracle.quantize_f32(h32[:, real], size2, scale2, zero2, out_bits)
+    assert np.array_equal(got, want32)
+    want64 = oracle.quantize(h64[:, real], size2, scale2.astype(np.float64), zero2, out_bits)
+    diff = np.abs(got.astype(int) - want64.astype(int))
+    assert diff.max() <= 1 and (diff[:, real] != 0).mean() <= 2e-3
+    # FC2 on those codes, original output order
+    W2 = (rng.normal(size=(C, H)) * 0.02).astype(np.float32)
+    w2_codes, s_w2, wsum2 = oracle.weight_quantize(W2, perm2, size2, None, C)
+    case2 = dict(perm=perm2, size=size2, scale=scale2, zero=zero2, w_codes=w2_codes, s_w=s_w2, wsum=wsum2, a=got,
+                 k_pad=k_pad2, bits=out_bits, M=M, N=C, n_pad=C)
+    d2 = _dev(case2)
+    d2["a"] = torch.from_numpy(packed).cuda()
+    y = _gemm(case2, d2)
+    want_y = _oracle_y(case2)
+    assert np.max(np.abs(y - want_y)) <= TOL * np.abs(want_y).max()
+
+
+def _workload_linear(site, li, rows):
+    """Oracle inputs and expected outputs of one LN -> linear site on sampled token rows."""
+    w = site.w
+    lin = w.linears[li]
+    W = workloads.weight_matrix(w, li, lin.n_out, w.hidden)
+    w_codes, s_w, wsum = oracle.weight_quantize(W, site.cal.perm, site.cal.size, None, lin.n_out)
+    y64 = oracle.reorder(oracle.layernorm(site.x[rows], site.gamma, site.beta, 1e-5), site.cal.perm)
+    a = oracle.quantize(y64, site.cal.size, site.cal.scale.astype(np.float64), site.cal.zero, site.bits)
+    return W, w_codes, s_w, wsum, a
+
+
+@pytest.mark.parametrize("name", ["opt-125m", "opt-1.3b"])
+def test_workload_configs_checked_in_full(name):
+    import torch
+    from paper_2304_01089_b200 import binding
+    site = Site(workloads.WORKLOADS[name])
+    w = site.w
+    rows = np.arange(w.tokens)
+    W, w_codes, s_w, wsum, a = _workload_linear(site, 0, rows)
+    N = w.linears[0].n_out
+    case = dict(perm=site.cal.perm, size=site.cal.size, scale=site.cal.scale, zero=site.cal.zero, w_codes=w_codes,
+                s_w=s_w, wsum=wsum, a=a, k_pad=a.shape[1], bits=site.bits, M=w.tokens, N=N, n_pad=N)
+    d = _dev(case)
+    # the library's own offline weight preparation must give the same bytes as the oracle's
+    packed_w, s_w_l, wsum_l = binding.weight_pack(d["L"], W)
+    assert np.array_equal(packed_w, oracle.pack_weights(w_codes)) and np.array_equal(s_w_l, s_w) and np.array_equal(wsum_l, wsum)
+    y = _gemm(case, d)
+    want = _oracle_y(case)
+    err = np.max(np.abs(y - want)) / np.abs(want).max()
+    print(f"{name}: max|dy|/max|y| = {err:.2e}")
+    assert err <= TOL
+    # the integer method agrees with de-quantise-then-matmul on the same codes (Appendix)
+    sub = slice(0, 8)
+    ref = oracle.dequant_matmul(a[sub], w_codes, site.cal.size, site.cal.scale.astype(np.float64), site.cal.zero, s_w)
+    assert np.max(np.abs(ref - want[sub])) <= 1e-10 * np.abs(want).max()

@@ -1,0 +1,123 @@
+"""CPU-side checks of the library boundary and of the host-side product code: the shared library
+loads and exports every declared symbol, argument validation, the packed-format helpers and the
+offline weight preparation against the oracle, and the numpy calibration against the oracle's."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2304_01089_b200 import build as lib_build
+from paper_2304_01089_b200 import calibration, workloads
+from helpers import random_layout_params
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def binding():
+    lib_build.build()
+    from paper_2304_01089_b200 import binding as b
+    return b
+
+
+def test_library_exports_every_declared_symbol(binding):
+    header = open(os.path.join(ROOT, "include", "rptq.h")).read()
+    declared = set(re.findall(r"\b(rptq_[a-z0-9_]+)\s*\(", header))
+    declared -= {"rptq_layout_t"}
+    assert declared == set(binding.EXPORTS)
+    lib = ctypes.CDLL(binding.LIB_PATH)
+    for name in declared:
+        assert hasattr(lib, name), name
+    assert binding.format_version() == 1
+    assert binding.status_string(-3) == "reorder index is not a bijection"
+
+
+def test_layout_validation_and_padded_offsets(binding):
+    rng = np.random.default_rng(0)
+    C, g, bits = 256, 6, 4
+    perm, size, scale, zero = random_layout_params(rng, C, g, bits)
+    L = binding.Layout(perm, size, scale, zero, bits)
+    off, k_pad = oracle.segment_offsets(size)
+    assert L.K_pad == k_pad and np.array_equal(L.seg_off, off) and L.row_bytes == k_pad // 2
+    off2, k_pad2 = calibration.segment_offsets(size)
+    assert k_pad2 == k_pad and np.array_equal(off2, off)
+    bad = perm.copy(); bad[3] = bad[4]
+    with pytest.raises(binding.RptqError) as e:
+        binding.Layout(bad, size, scale, zero, bits)
+    assert e.value.status == binding.ERR_NOT_BIJECTION
+    short = size.copy(); short[0] += 1
+    with pytest.raises(binding.RptqError) as e:
+        binding.Layout(perm, short, scale, zero, bits)
+    assert e.value.status == binding.ERR_NOT_BIJECTION
+    with pytest.raises(binding.RptqError) as e:
+        binding.Layout(perm, size, scale, zero, 5)
+    assert e.value.status == binding.ERR_UNSUPPORTED
+    neg = scale.copy(); neg[1] = 0.0
+    with pytest.raises(binding.RptqError) as e:
+        binding.Layout(perm, size, neg, zero, bits)
+    assert e.value.status == binding.ERR_INVALID_ARG
+    with pytest.raises(binding.RptqError) as e:
+        binding.Layout(np.arange(12, dtype=np.int32), [12], [1.0], [0], 4)
+    assert e.value.status == binding.ERR_UNSUPPORTED      # C not a multiple of 8
+
+
+@pytest.mark.parametrize("bits", [3, 4, 8])
+def test_packed_format_helpers_agree_with_the_oracle(binding, bits):
+    rng = np.random.default_rng(bits)
+    for k_pad in (128, 640, 1152):
+        codes = rng.integers(0, 1 << bits, size=(7, k_pad), dtype=np.uint8)
+        packed = binding.codes_pack_host(codes, bits)
+        assert np.array_equal(packed, oracle.pack(codes, bits))
+        assert np.array_equal(binding.codes_unpack_host(packed, k_pad, bits), codes)
+    w = rng.integers(-8, 8, size=(5, 256), dtype=np.int8)
+    assert np.array_equal(binding.weight_unpack_host(oracle.pack_weights(w), 256), w)
+
+
+def test_weight_pack_matches_the_oracle_bit_for_bit(binding):
+    rng = np.random.default_rng(5)
+    C, g, N, n_pad = 320, 7, 50, 64
+    perm, size, scale, zero = random_layout_params(rng, C, g, 4)
+    L = binding.Layout(perm, size, scale, zero, 4)
+    W = (rng.normal(size=(N, C)) * 0.02).astype(np.float32)
+    W[11] = 0
+    out_perm = rng.permutation(N).astype(np.int32)
+    for op in (None, out_perm):
+        packed, s_w, wsum = binding.weight_pack(L, W, op, n_pad)
+        w_codes, s_w_o, wsum_o = oracle.weight_quantize(W, perm, size, op, n_pad)
+        assert np.array_equal(packed, oracle.pack_weights(w_codes))
+        assert np.array_equal(s_w, s_w_o) and np.array_equal(wsum, wsum_o)
+    with pytest.raises(binding.RptqError):
+        binding.weight_pack(L, W, np.zeros(N, np.int32), n_pad)
+
+
+def test_numpy_calibration_agrees_with_the_oracle_calibration():
+    w = workloads.scaled(workloads.WORKLOADS["opt-125m"], tokens=16, calib_tokens=96)
+    gm, bt = workloads.ln_params(w)
+    x_cal = workloads.calib_tokens(w)
+    for bits in (3, 4, 8):
+        u = workloads.kmeans_draws(w, 0, w.clusters)
+        a = calibration.calibrate(x_cal, gm, bt, w.clusters, bits, u)
+        b = oracle.calibrate(x_cal, gm, bt, w.clusters, bits, u)
+        assert np.allclose(a.x_min, b.x_min, rtol=1e-12, atol=1e-12)
+        assert np.array_equal(a.perm, b.perm) and np.array_equal(a.size, b.size)
+        assert np.array_equal(a.zero, b.zero)
+        assert np.allclose(a.scale, b.scale.astype(np.float32), rtol=1e-6)
+    # Eq. 2 on the paper's example ranges
+    assert calibration.minmax_params(-100, -50, 4) == (3.125, 32)
+    assert calibration.minmax_params(80, 100, 4) == (1.25, -64)
+
+
+def test_workload_generators_are_seeded_and_shaped():
+    w = workloads.WORKLOADS["opt-125m"]
+    x1, x2 = workloads.test_tokens(w), workloads.test_tokens(w)
+    assert x1.dtype == np.float16 and x1.shape == (128, 768) and np.array_equal(x1, x2)
+    assert not np.array_equal(x1[:16], workloads.calib_tokens(w, 16))
+    gm, bt = workloads.ln_params(w)
+    assert gm.shape == (768,) and (gm.astype(np.float32) > 20).sum() >= 1
+    full = workloads.weight_matrix(w, 0, 3072, 768)
+    part = list(workloads.weight_rows(w, 0, 3072, 768, 1000, 1100))
+    assert np.array_equal(np.concatenate([b for _, b in part]), full[1000:1100])
+    assert abs(full.std() - 0.02) < 1e-3

@@ -1,0 +1,153 @@
+"""Parity of rptq_ln_reorder_quant (CUDA, through the C boundary) against the CPU oracle."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2304_01089_b200 import workloads
+from helpers import Site, random_layout_params
+
+pytestmark = pytest.mark.gpu
+
+EPS = 1e-5
+CANARY = 0xA5
+
+
+def _run(layout, x16, gamma16, beta16, want_y=True, ldx=None, stream=None):
+    import torch
+    from paper_2304_01089_b200 import binding
+    M, C = x16.shape
+    ldx = C if ldx is None else ldx
+    xd = torch.zeros((max(M, 1), ldx), dtype=torch.float16, device="cuda")
+    xd[:M, :C] = torch.from_numpy(x16).cuda()
+    gd, bd = torch.from_numpy(gamma16).cuda(), torch.from_numpy(beta16).cuda()
+    # one extra row of canary bytes behind the output
+    codes = torch.full((M + 1, layout.row_bytes), CANARY, dtype=torch.uint8, device="cuda")
+    y_dbg = torch.full((M + 1, C), float("nan"), dtype=torch.float32, device="cuda") if want_y else None
+    binding.ln_reorder_quant(layout, xd, gd, bd, EPS, codes, y_dbg, M=M, ldx=ldx, stream=stream)
+    torch.cuda.synchronize()
+    assert binding.get_device_status() == 0
+    codes_h = codes.cpu().numpy()
+    assert np.all(codes_h[M] == CANARY), "wrote past the last row"
+    y_h = None
+    if want_y:
+        y_h = y_dbg.cpu().numpy()
+        assert np.all(np.isnan(y_h[M]))
+        y_h = y_h[:M]
+    return codes_h[:M], y_h
+
+
+def _check_against_oracle(x16, gamma16, beta16, perm, size, scale32, zero, bits, packed, y_dbg, full_rate=0.9999):
+    M, C = x16.shape
+    _, k_pad = oracle.segment_offsets(size)
+    got = oracle.unpack(packed, k_pad, bits)
+    # (1) the decision, bit for bit, from the kernel's own fp32 LayerNorm outputs
+    want32 = oracle.quantize_f32(y_dbg, size, scale32, zero, bits)
+    assert np.array_equal(got, want32), "codes differ from the fp32-decision oracle on identical LN outputs"
+    assert np.array_equal(packed, oracle.pack(want32, bits)), "packed bytes differ from the documented format"
+    # (2) the whole step against the fp64 oracle
+    y64 = oracle.reorder(oracle.layernorm(x16, gamma16, beta16, EPS), perm)
+    want64 = oracle.quantize(y64, size, scale32.astype(np.float64), zero, bits)
+    diff = np.abs(got.astype(np.int16) - want64.astype(np.int16))
+    assert diff.max() <= 1, f"a code is off by {diff.max()}"
+    off, _ = oracle.segment_offsets(size)
+    real = np.concatenate([np.arange(off[c], off[c] + size[c]) for c in range(len(size))])
+    rate = 1.0 - diff[:, real].astype(bool).mean()
+    assert rate >= full_rate, f"only {rate:.6f} of the codes equal the fp64 oracle's"
+    # (3) the LayerNorm outputs themselves
+    tol = 2e-6 * np.abs(y64).max() + 1e-6
+    assert np.max(np.abs(y_dbg - y64)) <= 4 * tol
+    return rate
+
+
+@pytest.mark.parametrize("name", ["opt-125m", "opt-1.3b", "opt-6.7b", "opt-66b", "opt-175b"])
+def test_workload_configs_full_size(name):
+    site = Site(workloads.WORKLOADS[name])
+    L = site.layout()
+    packed, y_dbg = _run(L, site.x, site.gamma, site.beta)
+    rate = _check_against_oracle(site.x, site.gamma, site.beta, site.cal.perm, site.cal.size, site.cal.scale,
+                                 site.cal.zero, site.bits, packed, y_dbg)
+    print(f"{name}: {rate:.6f} of codes equal the fp64 oracle")
+    # same launch without the debug output and on another stream: identical bytes
+    import torch
+    s2 = torch.cuda.Stream()
+    packed2, _ = _run(L, site.x, site.gamma, site.beta, want_y=False, stream=s2)
+    assert np.array_equal(packed, packed2)
+
+
+@pytest.mark.parametrize("bits", [3, 4, 8])
+@pytest.mark.parametrize("M", [1, 2, 127, 129])
+def test_small_and_ragged_shapes_all_bit_widths(bits, M):
+    rng = np.random.default_rng(100 * bits + M)
+    C, g = 384, 5
+    perm, size, scale, zero = random_layout_params(rng, C, g, bits)
+    from paper_2304_01089_b200 import binding
+    L = binding.Layout(perm, size, scale, zero, bits)
+    x = (rng.normal(size=(M, C)) * 2).astype(np.float16)
+    gm = rng.lognormal(0, 0.5, C).astype(np.float16)
+    bt = rng.normal(size=C).astype(np.float16)
+    packed, y_dbg = _run(L, x, gm, bt, ldx=C + 24)
+    _check_against_oracle(x, gm, bt, perm, size, scale, zero, bits, packed, y_dbg, full_rate=0.999)
+
+
+@pytest.mark.parametrize("bits", [3, 4, 8])
+def test_degenerate_clusterings(bits):
+    from paper_2304_01089_b200 import binding
+    rng = np.random.default_rng(7 + bits)
+    C, M = 128, 33
+    x = rng.normal(size=(M, C)).astype(np.float16)
+    gm = rng.lognormal(0, 0.5, C).astype(np.float16)
+    bt = rng.normal(size=C).astype(np.float16)
+    # g = 1 with the identity index: plain LayerNorm + per-tensor quantisation
+    perm = np.arange(C, dtype=np.int32)
+    one = (perm, np.array([C], np.int32), np.array([0.21], np.float32), np.array([(1 << bits) // 2], np.int32))
+    # g = C: one channel per cluster (per-channel quantisation), K_pad = 32 * C
+    per_ch = (rng.permutation(C).astype(np.int32), np.ones(C, np.int32),
+              rng.uniform(0.05, 0.6, C).astype(np.float32), rng.integers(0, 1 << bits, C).astype(np.int32))
+    # many empty clusters
+    size = np.zeros(9, np.int32); size[2], size[7] = 100, 28
+    empty = (rng.permutation(C).astype(np.int32), size, rng.uniform(0.1, 0.5, 9).astype(np.float32),
+             rng.integers(0, 1 << bits, 9).astype(np.int32))
+    for perm_, size_, scale_, zero_ in (one, per_ch, empty):
+        L = binding.Layout(perm_, size_, scale_, zero_, bits)
+        packed, y_dbg = _run(L, x, gm, bt)
+        _check_against_oracle(x, gm, bt, perm_, size_, scale_, zero_, bits, packed, y_dbg, full_rate=0.999)
+
+
+def test_wide_rows_take_the_multi_unit_path_and_zero_tokens_launch_nothing():
+    from paper_2304_01089_b200 import binding
+    import torch
+    rng = np.random.default_rng(11)
+    C, g, bits, M = 16384, 40, 4, 9
+    perm, size, scale, zero = random_layout_params(rng, C, g, bits)
+    L = binding.Layout(perm, size, scale, zero, bits)
+    assert L.K_pad // 32 > 512
+    x = rng.normal(size=(M, C)).astype(np.float16)
+    gm = rng.lognormal(0, 0.5, C).astype(np.float16)
+    bt = rng.normal(size=C).astype(np.float16)
+    packed, y_dbg = _run(L, x, gm, bt)
+    _check_against_oracle(x, gm, bt, perm, size, scale, zero, bits, packed, y_dbg, full_rate=0.999)
+    codes = torch.full((4, L.row_bytes), CANARY, dtype=torch.uint8, device="cuda")
+    xd = torch.zeros((1, C), dtype=torch.float16, device="cuda")
+    binding.ln_reorder_quant(L, xd, torch.from_numpy(gm).cuda(), torch.from_numpy(bt).cuda(), EPS, codes, None, M=0)
+    torch.cuda.synchronize()
+    assert bool((codes == CANARY).all())
+
+
+def test_non_finite_inputs_still_give_in_range_codes():
+    from paper_2304_01089_b200 import binding
+    rng = np.random.default_rng(12)
+    C, bits = 256, 4
+    perm, size, scale, zero = random_layout_params(rng, C, 3, bits)
+    L = binding.Layout(perm, size, scale, zero, bits)
+    x = rng.normal(size=(4, C)).astype(np.float16)
+    x[1, 5] = np.inf
+    x[2, 9] = np.nan
+    gm = np.ones(C, np.float16); bt = np.zeros(C, np.float16)
+    packed, _ = _run(L, x, gm, bt)
+    got = oracle.unpack(packed, L.K_pad, bits)
+    assert got.max() <= 15
+    off, _ = oracle.segment_offsets(size)
+    pads = np.ones(L.K_pad, bool)
+    for c in range(3):
+        pads[off[c]:off[c] + size[c]] = False
+    assert not got[:, pads].any()

@@ -131,9 +131,16 @@ def test_fp32_decision_matches_fp64_decision_away_from_ties_and_its_own_definiti
     got = oracle.quantize_f32(y32, size, s32, z, 4)
     inv = (1.0 / s32.astype(np.float64)).astype(np.float32)
     off, _ = oracle.segment_offsets(size)
-    t = y32 * np.repeat(inv, size)[None, :]          # one fp32 multiply
-    assert t.dtype == np.float32
-    want = np.clip(np.rint(t) + np.repeat(z, size)[None, :].astype(np.float32), 0, 15).astype(np.uint8)
+    # exact product of the two fp32 numbers (fits fp64), rounded once to an integer
+    t = y32.astype(np.float64) * np.repeat(inv, size)[None, :].astype(np.float64)
+    want = np.clip(np.rint(t) + np.repeat(z, size)[None, :], 0, 15).astype(np.uint8)
+    # a product that sits just below a tie: rounding it to fp32 first would lift it onto the tie
+    # and change the code, the single rounding must not
+    y_t = np.array([[np.float32(2.5) * (1 - 2.0 ** -24)]], np.float32)
+    s_t = np.array([1.0], np.float32)
+    assert oracle.quantize_f32(y_t, [1], s_t, [0], 4)[0, 0] == 2
+    y_u = np.array([[np.float32(3.5)]], np.float32)
+    assert oracle.quantize_f32(y_u, [1], s_t, [0], 4)[0, 0] == 4
     cols = np.concatenate([np.arange(off[0], off[0] + 33), np.arange(off[1], off[1] + 31)])
     assert np.array_equal(got[:, cols], want)
     q64 = oracle.quantize(y32.astype(np.float64), size, s32.astype(np.float64), z, 4)
