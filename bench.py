@@ -1,0 +1,351 @@
+#!/usr/bin/env python
+"""Benchmark of the RPTQ hot path on B200: one step = LayerNorm+reorder+quantise followed by the
+cluster-segmented integer GEMM, for both LayerNorm sites of an OPT-66b-shaped decoder layer
+(hidden 9216: LN -> QKV 9216x27648 and LN -> FC1 9216x36864, 4096 tokens, 32 clusters, 3-bit
+activation codes, 4-bit weights), on seeded synthetic activations and weights.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints ONE JSON line. `value` is tera integer operations per second over the whole step
+(2*M*C*N per GEMM with the unpadded C, LayerNorm kernels included in the time). With N > 1
+(launched under torch.distributed.run) every rank runs its own batch of tokens against replicated
+weights: the path shards over tokens and has no exchange step, so there is no collective.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+WORKLOAD = "opt-66b"
+EPS = 1e-5
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            p = json.load(fh)
+        return dict(hbm=float(p["hbm_gbs"]), bf16_burst=float(p["bf16_tflops"]),
+                    bf16_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), source="measured")
+    return dict(hbm=6650.0, bf16_burst=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for name, v in zip(names, r[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def _sites(w):
+    """The two LayerNorm sites of the layer: (site workload, linear index into w.linears)."""
+    from paper_2304_01089_b200 import workloads
+    return [(workloads.scaled(w, name=w.name + "/ln1", seed=w.seed), 0),
+            (workloads.scaled(w, name=w.name + "/ln2", seed=w.seed + 1000), 1)]
+
+
+def _prepare_site(sw, li, n_tokens, torch, binding):
+    """Calibrate one site on the host, pack its weights, put everything on the device."""
+    from paper_2304_01089_b200 import calibration, workloads
+    gamma, beta = workloads.ln_params(sw)
+    cal = calibration.calibrate(workloads.calib_tokens(sw), gamma, beta, sw.clusters, sw.bits,
+                                workloads.kmeans_draws(sw, 0, sw.clusters), EPS)
+    L = binding.Layout(cal.perm, cal.size, cal.scale, cal.zero, sw.bits)
+    n_out = sw.linears[li].n_out
+    w_codes = np.empty((n_out, L.K_pad // 2), np.uint8)
+    s_w = np.empty(n_out, np.float32)
+    wsum = np.empty((sw.clusters, n_out), np.int32)
+    for lo, blk in workloads.weight_rows(sw, li, n_out, sw.hidden, chunk=4096):
+        wc, s, ws = binding.weight_pack(L, blk)
+        hi = lo + blk.shape[0]
+        w_codes[lo:hi], s_w[lo:hi], wsum[:, lo:hi] = wc, s, ws
+    x_host = torch.from_numpy(workloads.test_tokens(sw, n_tokens)).pin_memory()
+    return dict(sw=sw, L=L, cal=cal, n_out=n_out, gamma_h=gamma, beta_h=beta,
+                gamma=torch.from_numpy(gamma).cuda(), beta=torch.from_numpy(beta).cuda(),
+                w=torch.from_numpy(w_codes).cuda(), s_w=torch.from_numpy(s_w).cuda(), wsum=torch.from_numpy(wsum).cuda(),
+                bias=torch.from_numpy(workloads.bias_vector(sw, li, n_out)).cuda(),
+                x_host=x_host, x=x_host.cuda(),
+                codes=torch.empty((n_tokens, L.row_bytes), dtype=torch.uint8, device="cuda"),
+                y=torch.empty((n_tokens, n_out), dtype=torch.float16, device="cuda"),
+                y_host=torch.empty((n_tokens, n_out), dtype=torch.float16).pin_memory())
+
+
+def _step(sites, binding, M, events=None):
+    for i, s in enumerate(sites):
+        if events is not None:
+            events[i][0].record()
+        binding.ln_reorder_quant(s["L"], s["x"], s["gamma"], s["beta"], EPS, s["codes"], None, M=M)
+        if events is not None:
+            events[i][1].record()
+        binding.cluster_gemm(s["L"], s["codes"], M, s["w"], s["s_w"], s["wsum"], s["n_out"], s["y"],
+                             bias=s["bias"], y_dtype=binding.OUT_F16)
+        if events is not None:
+            events[i][2].record()
+
+
+def run_ours(args):
+    import torch
+    from paper_2304_01089_b200 import binding, workloads
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    w = workloads.WORKLOADS[WORKLOAD]
+    M, C = (args.tokens or w.tokens), w.hidden
+    # every rank processes its own batch of M tokens (weak scaling over tokens) against its own
+    # replica of the weights; all ranks draw the same seeded batch
+    sites = [_prepare_site(sw, li, M, torch, binding) for sw, li in _sites(w)]
+    ops_per_step = sum(2.0 * M * C * s["n_out"] for s in sites)
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(max(3, args.warmup)):
+        _step(sites, binding, M)
+    sync_all()
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.3)
+    ev = [[[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in sites] for _ in range(args.steps)]
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sync_all()
+    t0.record()
+    for k in range(args.steps):
+        _step(sites, binding, M, ev[k])
+    t1.record()
+    sync_all()
+    ms = t0.elapsed_time(t1)
+    clocks = sampler.stop()
+    status = binding.get_device_status()
+
+    ln_ms = [[ev[k][i][0].elapsed_time(ev[k][i][1]) for k in range(args.steps)] for i in range(len(sites))]
+    gm_ms = [[ev[k][i][1].elapsed_time(ev[k][i][2]) for k in range(args.steps)] for i in range(len(sites))]
+
+    # end to end through the C boundary with host buffers: H2D of the activations, D2H of the outputs
+    for _ in range(0 if args.no_e2e else 2):
+        for s in sites:
+            s["x"].copy_(s["x_host"], non_blocking=True)
+        _step(sites, binding, M)
+        for s in sites:
+            s["y_host"].copy_(s["y"], non_blocking=True)
+    sync_all()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e2e_steps = 0 if args.no_e2e else max(2, min(args.steps, 5))
+    e0.record()
+    for _ in range(e2e_steps):
+        for s in sites:
+            s["x"].copy_(s["x_host"], non_blocking=True)
+        _step(sites, binding, M)
+        for s in sites:
+            s["y_host"].copy_(s["y"], non_blocking=True)
+    e1.record()
+    sync_all()
+    e2e_ms = e0.elapsed_time(e1)
+
+    times = torch.tensor([ms, e2e_ms], dtype=torch.float64, device="cuda")
+    if dist is not None:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    ms, e2e_ms = float(times[0]), float(times[1])
+
+    if rank == 0:
+        peaks = _peaks()
+        int8_peak = 2.0 * peaks["bf16_sustained"]       # nominal int8 : bf16 dense ratio is 2
+        fc1 = sites[1]
+        fc1_ms = float(np.mean(gm_ms[1]))
+        fc1_ops = 2.0 * M * C * fc1["n_out"]
+        achieved = fc1_ops / (fc1_ms * 1e-3) / 1e12
+        ln_bytes = M * (2 * C + fc1["L"].row_bytes)
+        ln_gbs = ln_bytes / (float(np.mean(ln_ms[1])) * 1e-3) / 1e9
+        out = {
+            "metric": "LN+reorder+quant GB/s and cluster W4A4 GEMM TOPS (% roofline), 9216-hidden",
+            "value": world * ops_per_step * args.steps / (ms * 1e-3) / 1e12,
+            "unit": "TOPS",
+            "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
+            "ms_per_step": ms / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "int8xint8->int32 (3-bit activation codes, 4-bit weights), fp32 epilogue",
+            "data": "synthetic",
+            "config": {"workload": "opt-66b: 4096 tokens x hidden 9216, g=32, A3/W4; LN->QKV 27648 and LN->FC1 36864",
+                       "tokens_per_gpu": M, "full_size": M == w.tokens, "l2": "inputs larger than L2 (packed weights 127+169 MB, activations 2x75 MB per step)",
+                       "peaks": peaks["source"]},
+            "clocks": clocks,
+            "gpu_launches": 4 * args.steps,
+            "device_status": status,
+            "kernels": {
+                "ln_reorder_quant": {"ms": float(np.mean(ln_ms[1])), "GBps": ln_gbs, "frac_of_hbm": ln_gbs / peaks["hbm"],
+                                     "frac_of_8TBps": ln_gbs / 8000.0, "algorithmic_bytes": ln_bytes},
+                "cluster_gemm_qkv": {"ms": float(np.mean(gm_ms[0])),
+                                     "TOPS": 2.0 * M * C * sites[0]["n_out"] / (float(np.mean(gm_ms[0])) * 1e-3) / 1e12},
+                "cluster_gemm_fc1": {"ms": fc1_ms, "TOPS": achieved},
+            },
+            "roofline": {"bound": "tensor", "achieved": achieved, "peak": int8_peak, "unit": "TOP/s",
+                         "frac": achieved / int8_peak, "traffic": None,
+                         "kernel": "cluster_gemm_kernel<3> 4096x9216x36864",
+                         "peak_note": f"2 x bf16 sustained ({peaks['source']})"},
+            "e2e": None if args.no_e2e else {"value": world * ops_per_step * e2e_steps / (e2e_ms * 1e-3) / 1e12, "unit": "TOPS",
+                    "h2d_bytes_per_step": int(sum(s["x_host"].numel() * 2 for s in sites)),
+                    "d2h_bytes_per_step": int(sum(s["y_host"].numel() * 2 for s in sites))},
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            out["cpu_baseline"] = cpu_baseline(sites[1], M)
+        print(json.dumps(out), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def _oracle_sample(site, rows_ln: int, rows_gemm: int):
+    """One bounded pass of the oracle over a sample of the FC1 site: LayerNorm+reorder+quantise on
+    `rows_ln` tokens, the cluster GEMM on `rows_gemm` of them against all output channels."""
+    import oracle
+    from paper_2304_01089_b200 import workloads
+    sw, cal = site["sw"], site["cal"]
+    x = workloads.test_tokens(sw, rows_ln)
+    n_out = site["n_out"]
+    w_packed = site["w"].cpu().numpy() if hasattr(site["w"], "cpu") else site["w"]
+    w_codes = oracle.unpack_weights(w_packed, site["L"].K_pad)
+    s_w = site["s_w"].cpu().numpy() if hasattr(site["s_w"], "cpu") else site["s_w"]
+    wsum = site["wsum"].cpu().numpy() if hasattr(site["wsum"], "cpu") else site["wsum"]
+    t0 = time.perf_counter()
+    y = oracle.reorder(oracle.layernorm(x, site["gamma_h"], site["beta_h"], EPS), cal.perm)
+    codes = oracle.quantize(y, cal.size, cal.scale.astype(np.float64), cal.zero, sw.bits)
+    oracle.pack(codes, sw.bits)
+    t1 = time.perf_counter()
+    oracle.cluster_gemm(codes[:rows_gemm], w_codes, cal.size, cal.scale.astype(np.float64), cal.zero, s_w, wsum)
+    t2 = time.perf_counter()
+    ops = 2.0 * rows_gemm * sw.hidden * n_out
+    return ops, t2 - t0, t1 - t0, t2 - t1
+
+
+def cpu_baseline(site, M):
+    rows_ln, rows_gemm = 256, 8
+    ops, total, t_ln, t_gemm = _oracle_sample(site, rows_ln, rows_gemm)
+    # scale the sample so that it takes roughly 10-30 s of CPU work
+    if t_gemm < 5.0:
+        rows_gemm = int(min(M, max(rows_gemm, rows_gemm * 15.0 / max(t_gemm, 1e-3))))
+        rows_ln = max(rows_ln, rows_gemm)
+        ops, total, t_ln, t_gemm = _oracle_sample(site, rows_ln, rows_gemm)
+    return {"value": ops / total / 1e12, "unit": "TOPS", "cores": len(os.sched_getaffinity(0)), "kind": "oracle",
+            "sample": f"FC1 site: LN+reorder+quant of {rows_ln} tokens ({t_ln:.2f} s) + cluster GEMM of {rows_gemm} tokens "
+                      f"x 9216 x 36864 ({t_gemm:.2f} s), OpenMP over tokens"}
+
+
+def run_reference(args):
+    """The reference arm is the CPU oracle as it stands, on the machine's host cores (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    from paper_2304_01089_b200 import calibration, workloads
+    import oracle
+    w = workloads.WORKLOADS[WORKLOAD]
+    sw, li = _sites(w)[1]
+    gamma, beta = workloads.ln_params(sw)
+    cal = calibration.calibrate(workloads.calib_tokens(sw), gamma, beta, sw.clusters, sw.bits,
+                                workloads.kmeans_draws(sw, 0, sw.clusters), EPS)
+    n_out = sw.linears[li].n_out
+    W = workloads.weight_matrix(sw, li, n_out, sw.hidden)
+    w_codes, s_w, wsum = oracle.weight_quantize(W, cal.perm, cal.size, None, n_out)
+    _, k_pad = oracle.segment_offsets(cal.size)
+
+    class _L:
+        K_pad = k_pad
+    site = dict(sw=sw, cal=cal, n_out=n_out, gamma_h=gamma, beta_h=beta, w=oracle.pack_weights(w_codes), s_w=s_w,
+                wsum=wsum, L=_L)
+    rows_ln, rows_gemm = 64, 4
+    warm = max(1, min(args.warmup, 2))
+    for _ in range(warm):
+        _oracle_sample(site, rows_ln, rows_gemm)
+    steps = max(1, min(args.steps, 5))
+    t = 0.0
+    ops = 0.0
+    for _ in range(steps):
+        o, total, _, _ = _oracle_sample(site, rows_ln, rows_gemm)
+        ops += o
+        t += total
+    value = ops / t / 1e12
+    cores = len(os.sched_getaffinity(0))
+    sample = f"per step: FC1 site, LN+reorder+quant of {rows_ln} tokens + cluster GEMM of {rows_gemm} tokens x 9216 x 36864"
+    print(json.dumps({
+        "impl": "reference",
+        "metric": "LN+reorder+quant GB/s and cluster W4A4 GEMM TOPS (% roofline), 9216-hidden",
+        "value": value, "unit": "TOPS", "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": steps, "warmup": warm,
+        "ms_per_step": t / steps * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "int64 accumulate, fp64 epilogue (CPU oracle)", "data": "synthetic",
+        "config": {"workload": "opt-66b: 4096 tokens x hidden 9216, g=32, A3/W4; LN->FC1 36864 (bounded sample per step)"},
+        "cpu_baseline": {"value": value, "unit": "TOPS", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "TOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=40)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", choices=("ours", "reference"), default="ours")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--tokens", type=int, default=None, help="tokens per GPU (default: the workload's 4096); smaller values are for profiler captures")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
