@@ -33,12 +33,12 @@ class RptqError(RuntimeError):
         super().__init__(f"{where}: {status_string(status)} ({status})")
 
 
-def _load() -> C.CDLL:
-    if not os.path.exists(LIB_PATH):
+def _load(path: str = LIB_PATH) -> C.CDLL:
+    if not os.path.exists(path):
         raise ImportError(
-            f"{LIB_PATH} is missing: build it with `python -m paper_2304_01089_b200.build` "
+            f"{path} is missing: build it with `python -m paper_2304_01089_b200.build` "
             "(nvcc, sm_100a). There is no CPU or PyTorch fallback.")
-    lib = C.CDLL(LIB_PATH)
+    lib = C.CDLL(path)
     vp, i32, i64, f32 = C.c_void_p, C.c_int, C.c_int64, C.c_float
     lib.rptq_layout_create.argtypes = [C.POINTER(vp), i32, i32, i32, vp, vp, vp, vp]
     lib.rptq_layout_query.argtypes = [vp, C.POINTER(i32), C.POINTER(i64), vp]

@@ -35,7 +35,7 @@ constexpr int UNPACK_WARP0 = 4, N_UNPACK_WARPS = 4;
 constexpr int EPI_WARP0 = 8, N_EPI_WARPS = 8;
 constexpr int A8_BYTES = TILE_M * KBLK, W8_BYTES = TILE_N * KBLK;     // 16 KB, 32 KB
 constexpr int WP_BYTES = TILE_N * KBLK / 2;                           // 16 KB packed weights per stage
-constexpr uint64_t WAIT_BUDGET_NS = 2000000000ull;
+constexpr long long WAIT_BUDGET_CYCLES = 4000000000ll;   // about two seconds at the SM clock
 
 __host__ __device__ constexpr int ap_bytes(int bits) { return TILE_M * KBLK * bits / 8; }
 
@@ -101,25 +101,26 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-__device__ __forceinline__ uint64_t globaltimer_ns()
+// Bounded wait. Returns false when the budget ran out or another role already gave up. The common
+// case (the phase has already completed, or completes within a few polls) touches no timer; the
+// budget is counted on the SM's cycle counter, read once per batch of polls.
+__device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, bool heed_abort)
 {
-    uint64_t t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-// Bounded wait. Returns false when the budget ran out or another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, bool heed_abort = true)
-{
-#pragma unroll 1
-    for (int i = 0; i < 128; ++i)
-        if (mbar_try_wait(bar, parity)) return true;
-    const uint64_t t0 = globaltimer_ns();
+    const long long t0 = clock64();
 #pragma unroll 1
     while (true) {
-        if (mbar_try_wait(bar, parity)) return true;
+#pragma unroll 1
+        for (int i = 0; i < 1024; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
         if (heed_abort && *abort_flag) return false;
-        if (globaltimer_ns() - t0 > WAIT_BUDGET_NS) { *abort_flag = 1; return false; }
+        if (clock64() - t0 > WAIT_BUDGET_CYCLES) { *abort_flag = 1; return false; }
     }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, bool heed_abort = true)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, abort_flag, heed_abort);
 }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar)
 {
@@ -185,16 +186,6 @@ __device__ __forceinline__ uint32_t lds32(uint32_t addr)
     return v;
 }
 
-// One unpack work item: 32 codes of one operand row -> 32 bytes at K offset 32*unit of that row
-// in the swizzled tile (16-byte chunk j of row r lives at chunk position j ^ (r & 7)).
-__device__ __forceinline__ void store_item(uint32_t tile, int row, int unit, const uint32_t (&o)[8])
-{
-    const uint32_t base = tile + row * 128;
-    const int sw = row & 7;
-    sts128(base + (((2 * unit) ^ sw) << 4), o[0], o[1], o[2], o[3]);
-    sts128(base + (((2 * unit + 1) ^ sw) << 4), o[4], o[5], o[6], o[7]);
-}
-
 template <int BITS>
 __global__ void __launch_bounds__(THREADS, 1)
 cluster_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w, const Params p)
@@ -250,7 +241,7 @@ cluster_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
     // The register file is re-partitioned by warpgroup (the epilogue holds 128 running sums per
     // thread); each setmaxnreg is executed by the four warps of its group at one place.
     if (warp < UNPACK_WARP0) {
-      asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
+      asm volatile("setmaxnreg.dec.sync.aligned.u32 24;");
       if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
@@ -277,40 +268,56 @@ cluster_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
       } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
+            // This lane is a single thread of dependent instructions, so the loop is kept short:
+            // stage descriptors are built once, a K block's four step flags come as one word, and a
+            // block that lies inside one cluster issues its four MMAs without any test.
             uint32_t n_kb_done = 0, n_seg_done = 0;
             bool ok = true;
+            const uint64_t a_desc0 = smem_desc_sw128(smem_base), w_desc0 = smem_desc_sw128(smem_base + A8_BYTES);
+            const uint32_t* flags4 = reinterpret_cast<const uint32_t*>(s_flags);
+            uint32_t d_tmem = tmem_base;
             for (int t = blockIdx.x; t < p.n_tiles && ok; t += gridDim.x) {
                 for (int kb = 0; kb < p.n_kb && ok; ++kb, ++n_kb_done) {
                     const int s = n_kb_done % N_U;
                     if (!mbar_wait(bar(B_UFULL + s), (n_kb_done / N_U) & 1, s_abort)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t a_tile = smem_base + s * SL.u_stage, w_tile = a_tile + A8_BYTES;
-#pragma unroll 1
-                    for (int j = 0; j < 4; ++j) {
-                        const uint8_t f = s_flags[kb * 4 + j];
-                        if (f & STEP_SKIP) continue;
-                        const uint32_t buf = n_seg_done & 1;
-                        if (f & STEP_FIRST) {
-                            if (!mbar_wait(bar(B_ACCEMPTY + buf), ((n_seg_done >> 1) & 1) ^ 1, s_abort)) { ok = false; break; }
-                            tc_fence_after();
+                    // the start-address field counts 16-byte units: one stage further, 32 bytes per step
+                    const uint64_t ad = a_desc0 + (uint64_t)(s * (SL.u_stage >> 4)), wd = w_desc0 + (uint64_t)(s * (SL.u_stage >> 4));
+                    const uint32_t f4 = flags4[kb];
+                    if (f4 == 0) {
+                        tc_mma_i8(d_tmem, ad, wd, kInstrDesc, 1u);
+                        tc_mma_i8(d_tmem, ad + 2, wd + 2, kInstrDesc, 1u);
+                        tc_mma_i8(d_tmem, ad + 4, wd + 4, kInstrDesc, 1u);
+                        tc_mma_i8(d_tmem, ad + 6, wd + 6, kInstrDesc, 1u);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const uint32_t f = (f4 >> (8 * j)) & 0xFFu;
+                            if (f & STEP_SKIP) continue;
+                            if (f & STEP_FIRST) {
+                                if (!mbar_wait(bar(B_ACCEMPTY + (n_seg_done & 1)), ((n_seg_done >> 1) & 1) ^ 1, s_abort)) { ok = false; break; }
+                                tc_fence_after();
+                            }
+                            tc_mma_i8(d_tmem, ad + 2 * j, wd + 2 * j, kInstrDesc, (f & STEP_FIRST) ? 0u : 1u);
+                            if (f & STEP_LAST) {
+                                tc_commit(bar(B_ACCFULL + (n_seg_done & 1)));
+                                ++n_seg_done;
+                                d_tmem = tmem_base + (n_seg_done & 1) * TILE_N;
+                            }
                         }
-                        tc_mma_i8(tmem_base + buf * TILE_N, smem_desc_sw128(a_tile + j * 32), smem_desc_sw128(w_tile + j * 32),
-                                  kInstrDesc, (f & STEP_FIRST) ? 0u : 1u);
-                        if (f & STEP_LAST) { tc_commit(bar(B_ACCFULL + buf)); ++n_seg_done; }
                     }
                     tc_commit(bar(B_UEMPTY + s));      // the stage may be overwritten once these MMAs have read it
                 }
             }
             if (!ok) {
                 tc_commit(bar(B_DRAIN));
-                const uint64_t t0 = globaltimer_ns();
-                while (!mbar_try_wait(bar(B_DRAIN), 0) && globaltimer_ns() - t0 < WAIT_BUDGET_NS) {}
+                mbar_wait(bar(B_DRAIN), 0, s_abort, false);
             }
         }
       }   // warps 2 and 3 only fill the first warpgroup
     } else if (warp < EPI_WARP0) {
         // ------------------------------------------------------------ unpack warps
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 88;");
         const int ut = tid - UNPACK_WARP0 * 32;      // 0..127
         uint32_t n_done = 0;
         bool ok = true;
@@ -322,34 +329,45 @@ cluster_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
             tc_fence_after();
             const uint32_t pa = smem_base + SL.off_p + sp * SL.p_stage, pw = pa + AP_BYTES;
             const uint32_t a_tile = smem_base + su * SL.u_stage, w_tile = a_tile + A8_BYTES;
-            // activations: 128 rows x 4 units
+            // All packed words of my 12 items first (independent loads), then unpack and store.
+            // Item i of this thread is row (ut >> 2) + 32 i, unit ut & 3, so its two chunk positions
+            // in the swizzled row are the same for every i.
+            uint32_t pa_w[4][BITS], pw_w[8][4];
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const int item = ut + i * 128;
-                uint32_t pk[BITS], o[8];
                 if constexpr (BITS == 4) {
                     const uint4 v = lds128(pa + item * 16);
-                    pk[0] = v.x; pk[1] = v.y; pk[2] = v.z; pk[3] = v.w;
+                    pa_w[i][0] = v.x; pa_w[i][1] = v.y; pa_w[i][2] = v.z; pa_w[i][3] = v.w;
                 } else if constexpr (BITS == 3) {
 #pragma unroll
-                    for (int j = 0; j < 3; ++j) pk[j] = lds32(pa + item * 12 + j * 4);
+                    for (int j = 0; j < 3; ++j) pa_w[i][j] = lds32(pa + item * 12 + j * 4);
                 } else {
                     const uint4 v0 = lds128(pa + item * 32), v1 = lds128(pa + item * 32 + 16);
-                    pk[0] = v0.x; pk[1] = v0.y; pk[2] = v0.z; pk[3] = v0.w;
-                    pk[4] = v1.x; pk[5] = v1.y; pk[6] = v1.z; pk[7] = v1.w;
+                    pa_w[i][0] = v0.x; pa_w[i][1] = v0.y; pa_w[i][2] = v0.z; pa_w[i][3] = v0.w;
+                    pa_w[i][4] = v1.x; pa_w[i][5] = v1.y; pa_w[i][6] = v1.z; pa_w[i][7] = v1.w;
                 }
-                unpack_act32<BITS>(pk, o);
-                store_item(a_tile, item >> 2, item & 3, o);
             }
-            // weights: 256 rows x 4 units
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
-                const int item = ut + i * 128;
-                const uint4 v = lds128(pw + item * 16);
-                const uint32_t pk[4] = {v.x, v.y, v.z, v.w};
+                const uint4 v = lds128(pw + (ut + i * 128) * 16);
+                pw_w[i][0] = v.x; pw_w[i][1] = v.y; pw_w[i][2] = v.z; pw_w[i][3] = v.w;
+            }
+            const int row0 = ut >> 2, unit = ut & 3, sw = row0 & 7;
+            const uint32_t off0 = row0 * 128 + (((2 * unit) ^ sw) << 4), off1 = row0 * 128 + (((2 * unit + 1) ^ sw) << 4);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
                 uint32_t o[8];
-                unpack_w32_x16(pk, o);
-                store_item(w_tile, item >> 2, item & 3, o);
+                unpack_act32<BITS>(pa_w[i], o);
+                sts128(a_tile + off0 + i * 4096, o[0], o[1], o[2], o[3]);
+                sts128(a_tile + off1 + i * 4096, o[4], o[5], o[6], o[7]);
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                uint32_t o[8];
+                unpack_w32_x16(pw_w[i], o);
+                sts128(w_tile + off0 + i * 4096, o[0], o[1], o[2], o[3]);
+                sts128(w_tile + off1 + i * 4096, o[4], o[5], o[6], o[7]);
             }
             fence_proxy_async();          // make the generic-proxy stores visible to the tensor core
             __syncwarp();
@@ -530,7 +548,7 @@ static int launch(const CUtensorMap& tm_a, const CUtensorMap& tm_w, const Params
     cudaFuncAttributes attr;
     if (cudaFuncGetAttributes(&attr, fn) != cudaSuccess) return RPTQ_ERR_CUDA;
     // the register re-partition inside the kernel (setmaxnreg) assumes this pool; refuse to launch otherwise
-    if (attr.numRegs * THREADS < 40 * 128 + 64 * 128 + 200 * 256) return RPTQ_ERR_UNSUPPORTED;
+    if (attr.numRegs * THREADS < 24 * 128 + 88 * 128 + 200 * 256) return RPTQ_ERR_UNSUPPORTED;
     if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return RPTQ_ERR_CUDA;
     cluster_gemm_kernel<BITS><<<grid, THREADS, smem, st>>>(tm_a, tm_w, p);
     return cudaGetLastError() == cudaSuccess ? RPTQ_OK : RPTQ_ERR_CUDA;
