@@ -88,6 +88,9 @@ int rptq_layout_create(rptq_layout_t** out, int C, int g, int bits,
 /* Sizes of the padded layout. Any output pointer may be NULL. seg_offset_out receives g+1 ints. */
 int rptq_layout_query(const rptq_layout_t* L, int* K_pad, int64_t* row_bytes, int32_t* seg_offset_out);
 
+/* padded_index[K_pad]: the original channel held by each padded position, -1 for pad positions. */
+int rptq_layout_padded_index(const rptq_layout_t* L, int32_t* padded_index);
+
 /* Frees the handle and its device tables. Work that uses it must have completed. NULL is OK. */
 int rptq_layout_destroy(rptq_layout_t* L);
 
@@ -116,8 +119,12 @@ int rptq_ln_reorder_quant(const rptq_layout_t* L, const void* x, int64_t ldx, co
  * orientation (Y = X W^T). Weights are quantised round-to-nearest, symmetric, one scale per output
  * channel (the paper uses GPTQ, which needs a trained model's statistics):
  *   s_w[n] = max_k |W[n][k]| / 7 (1 if the row is zero), w_q = clamp(rne(W / s_w), -8, 7), in fp32.
- *   out_perm      NULL, or host int32 [N]: output row r is original row out_perm[r]
- *   N_pad         >= N; rows N..N_pad-1 are zero with s_w = 1
+ *   N_pad         >= N, the number of output rows written
+ *   out_perm      NULL: output row r is original row r for r < N and a zero row (s_w = 1) beyond.
+ *                 Otherwise host int32 [N_pad]: output row r is original row out_perm[r], or a zero
+ *                 row where out_perm[r] < 0; no original row may appear twice. With the array that
+ *                 rptq_layout_padded_index gives for the next site, the output channels come out in
+ *                 that site's padded cluster order and rptq_cluster_gemm can re-quantise them in place.
  *   w_codes_host  host, N_pad rows of K_pad/2 bytes (packed signed nibbles, padded segment layout)
  *   s_w           host fp32 [N_pad]
  *   wsum          host int32 [g][N_pad]: Wsum_c[r] = sum of w_q over the channels of cluster c

@@ -185,6 +185,10 @@ def weight_quantize(W: np.ndarray, perm, size, out_perm=None, n_pad: Optional[in
     g = size.shape[0]
     _, k_pad = segment_offsets(size)
     op = None if out_perm is None else _arr(out_perm, np.int32)
+    if op is not None:
+        if n_pad == N and op.shape[0] != N:
+            n_pad = int(op.shape[0])
+        assert op.shape[0] == n_pad, "out_perm has one entry per output row"
     w_codes = np.empty((n_pad, k_pad), np.int8)
     s_w = np.empty(n_pad, np.float32)
     wsum = np.empty((g, n_pad), np.int32)

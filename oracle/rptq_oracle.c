@@ -426,8 +426,10 @@ void orc_unpack_weight_codes(const uint8_t* packed, int64_t N, int32_t K_pad, in
  * per output channel (the paper itself uses GPTQ, which needs model Hessians):
  *     s_w[n] = max_k |W[n,k]| / 7  (1 when the row is zero),  w_q = clamp(rne(W / s_w), -8, 7),
  * both evaluated in IEEE fp32 because they decide integers and the library decides them in
- * fp32. Output row r of w_codes is original row out_perm[r] (identity when out_perm is NULL);
- * rows N..N_pad-1 are zero with s_w = 1. Column layout: padded cluster segments, pads = 0.
+ * fp32. "Rows (dimension C2) based on the output activation reorder index": output row r of
+ * w_codes is original row out_perm[r] for r < N_pad, or a zero row with s_w = 1 where
+ * out_perm[r] < 0 (the pad positions of the next site's padded layout); with out_perm NULL, row r
+ * is original row r for r < N and zero beyond. Column layout: padded cluster segments, pads = 0.
  * wsum[c][r] = sum over the real channels of cluster c of w_q. */
 void orc_weight_quantize(const float* W, int64_t N, int C, int g, const int32_t* perm,
                          const int32_t* size, const int32_t* out_perm, int64_t N_pad, int32_t K_pad,
@@ -441,8 +443,9 @@ void orc_weight_quantize(const float* W, int64_t N, int C, int g, const int32_t*
         for (int c = 0; c < g; ++c) wsum[(int64_t)c * N_pad + r] = 0;
     }
 #pragma omp parallel for schedule(static)
-    for (int64_t r = 0; r < N; ++r) {
-        int64_t n = out_perm ? out_perm[r] : r;
+    for (int64_t r = 0; r < N_pad; ++r) {
+        int64_t n = out_perm ? out_perm[r] : (r < N ? r : -1);
+        if (n < 0) continue;
         const float* wr = W + n * C;
         float amax = 0.0f;
         for (int kk = 0; kk < C; ++kk) {

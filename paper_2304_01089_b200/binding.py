@@ -23,7 +23,7 @@ EXPORTS = (
     "rptq_layout_create", "rptq_layout_query", "rptq_layout_destroy", "rptq_ln_reorder_quant",
     "rptq_weight_pack", "rptq_cluster_gemm", "rptq_cluster_gemm_debug_acc", "rptq_codes_unpack_host",
     "rptq_codes_pack_host", "rptq_weight_unpack_host", "rptq_get_device_status", "rptq_status_string",
-    "rptq_format_version",
+    "rptq_format_version", "rptq_layout_padded_index",
 )
 
 
@@ -43,6 +43,7 @@ def _load(path: str = LIB_PATH) -> C.CDLL:
     lib.rptq_layout_create.argtypes = [C.POINTER(vp), i32, i32, i32, vp, vp, vp, vp]
     lib.rptq_layout_query.argtypes = [vp, C.POINTER(i32), C.POINTER(i64), vp]
     lib.rptq_layout_destroy.argtypes = [vp]
+    lib.rptq_layout_padded_index.argtypes = [vp, vp]
     lib.rptq_ln_reorder_quant.argtypes = [vp, vp, i64, vp, vp, f32, i32, vp, vp, vp]
     lib.rptq_weight_pack.argtypes = [vp, vp, i32, vp, i32, vp, vp, vp]
     lib.rptq_cluster_gemm.argtypes = [vp, vp, i32, vp, vp, vp, i64, vp, i32, i32, vp, vp, i32, i64, vp]
@@ -121,6 +122,12 @@ class Layout:
             raise ValueError("layout was destroyed")
         return self._h
 
+    def padded_index(self) -> np.ndarray:
+        """int32 [K_pad]: original channel at each padded position, -1 at pads."""
+        out = np.empty(self.K_pad, np.int32)
+        _check(_lib.rptq_layout_padded_index(self.handle, _np_ptr(out)), "rptq_layout_padded_index")
+        return out
+
     def destroy(self) -> None:
         if getattr(self, "_h", None) is not None:
             _lib.rptq_layout_destroy(self._h)
@@ -153,6 +160,10 @@ def weight_pack(layout_in: Layout, W: np.ndarray, out_perm=None, n_pad: Optional
         raise ValueError("W must be [N][C] with C the layout's channel count")
     n_pad = N if n_pad is None else int(n_pad)
     op = None if out_perm is None else np.ascontiguousarray(out_perm, dtype=np.int32)
+    if op is not None:
+        n_pad = int(op.shape[0]) if n_pad == N and op.shape[0] != N else n_pad
+        if op.shape[0] != n_pad:
+            raise ValueError("out_perm must have one entry per output row (N_pad)")
     w_codes = np.empty((n_pad, layout_in.K_pad // 2), np.uint8)
     s_w = np.empty(n_pad, np.float32)
     wsum = np.empty((layout_in.g, n_pad), np.int32)

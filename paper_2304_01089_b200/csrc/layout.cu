@@ -213,6 +213,16 @@ int rptq_layout_query(const rptq_layout_t* L, int* K_pad, int64_t* row_bytes, in
     return RPTQ_OK;
 }
 
+int rptq_layout_padded_index(const rptq_layout_t* L, int32_t* padded_index)
+{
+    if (!L || !padded_index) return RPTQ_ERR_INVALID_ARG;
+    for (int p = 0; p < L->K_pad; ++p) padded_index[p] = -1;
+    int j = 0;
+    for (int c = 0; c < L->g; ++c)
+        for (int i = 0; i < L->size[c]; ++i, ++j) padded_index[L->seg_off[c] + i] = L->perm[j];
+    return RPTQ_OK;
+}
+
 int rptq_layout_destroy(rptq_layout_t* L)
 {
     if (!L) return RPTQ_OK;
@@ -264,8 +274,9 @@ int rptq_weight_pack(const rptq_layout_t* Lin, const float* W_host, int N, const
     const int C = Lin->C, g = Lin->g, K_pad = Lin->K_pad;
     if (out_perm) {
         std::vector<uint8_t> seen((size_t)N, 0);
-        for (int r = 0; r < N; ++r) {
-            if (out_perm[r] < 0 || out_perm[r] >= N || seen[out_perm[r]]) return RPTQ_ERR_NOT_BIJECTION;
+        for (int r = 0; r < N_pad; ++r) {
+            if (out_perm[r] < 0) continue;
+            if (out_perm[r] >= N || seen[out_perm[r]]) return RPTQ_ERR_NOT_BIJECTION;
             seen[out_perm[r]] = 1;
         }
     }
@@ -279,8 +290,9 @@ int rptq_weight_pack(const rptq_layout_t* Lin, const float* W_host, int N, const
         for (int r = 0; r < N_pad; ++r) {
             std::memset(row.data(), 0, (size_t)K_pad);
             float s = 1.0f;
-            if (r < N) {
-                const float* w = W_host + (int64_t)(out_perm ? out_perm[r] : r) * C;
+            const int src_row = out_perm ? out_perm[r] : (r < N ? r : -1);
+            if (src_row >= 0) {
+                const float* w = W_host + (int64_t)src_row * C;
                 float amax = 0.0f;
                 for (int k = 0; k < C; ++k) amax = fmaxf(amax, fabsf(w[k]));
                 if (!std::isfinite(amax)) failed = 1;

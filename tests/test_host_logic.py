@@ -83,14 +83,24 @@ def test_weight_pack_matches_the_oracle_bit_for_bit(binding):
     L = binding.Layout(perm, size, scale, zero, 4)
     W = (rng.normal(size=(N, C)) * 0.02).astype(np.float32)
     W[11] = 0
-    out_perm = rng.permutation(N).astype(np.int32)
+    out_perm = np.full(n_pad, -1, np.int32)
+    out_perm[np.sort(rng.choice(n_pad, size=N, replace=False))] = rng.permutation(N)
     for op in (None, out_perm):
         packed, s_w, wsum = binding.weight_pack(L, W, op, n_pad)
         w_codes, s_w_o, wsum_o = oracle.weight_quantize(W, perm, size, op, n_pad)
         assert np.array_equal(packed, oracle.pack_weights(w_codes))
         assert np.array_equal(s_w, s_w_o) and np.array_equal(wsum, wsum_o)
     with pytest.raises(binding.RptqError):
-        binding.weight_pack(L, W, np.zeros(N, np.int32), n_pad)
+        binding.weight_pack(L, W, np.zeros(n_pad, np.int32), n_pad)
+    # the padded index of a layout is what places a previous layer's rows for re-quantisation
+    idx = L.padded_index()
+    off, _ = oracle.segment_offsets(size)
+    want = np.full(L.K_pad, -1, np.int32)
+    j = 0
+    for c in range(g):
+        want[off[c]:off[c] + size[c]] = perm[j:j + size[c]]
+        j += size[c]
+    assert np.array_equal(idx, want)
 
 
 def test_numpy_calibration_agrees_with_the_oracle_calibration():

@@ -283,11 +283,13 @@ def test_weight_quantise_per_output_channel_symmetric_and_wsum_brute_force():
     W[3] = 0
     size = np.array([20, 0, 50, 26], np.int32)
     perm = r.permutation(Cn).astype(np.int32)
-    out_perm = r.permutation(N).astype(np.int32)
+    out_perm = np.full(16, -1, np.int32)                       # rows 2, 5, 9.. of the output are zero pads
+    slots = np.sort(r.choice(16, size=N, replace=False))
+    out_perm[slots] = r.permutation(N)
     w_codes, s_w, wsum = oracle.weight_quantize(W, perm, size, out_perm, n_pad=16)
     off, k_pad = oracle.segment_offsets(size)
     assert w_codes.shape == (16, k_pad) and wsum.shape == (4, 16)
-    for rrow in range(N):
+    for rrow in slots:
         src = W[out_perm[rrow]]
         amax = np.abs(src).max()
         s = np.float32(amax) / np.float32(7) if amax > 0 else np.float32(1)
@@ -301,8 +303,12 @@ def test_weight_quantise_per_output_channel_symmetric_and_wsum_brute_force():
             assert not seg[size[c]:].any()
             assert wsum[c, rrow] == int(q[perm[j:j + size[c]]].astype(int).sum())
             j += size[c]
-    assert not w_codes[N:].any() and np.all(s_w[N:] == 1) and not wsum[:, N:].any()
+    pads = np.setdiff1d(np.arange(16), slots)
+    assert not w_codes[pads].any() and np.all(s_w[pads] == 1) and not wsum[:, pads].any()
     assert np.all(s_w[list(out_perm).index(3)] == 1)
+    # without an output index: identity rows, zero rows beyond N
+    w2, s2, ws2 = oracle.weight_quantize(W, perm, size, None, n_pad=16)
+    assert np.array_equal(w2[out_perm[slots]], w_codes[slots]) and not w2[N:].any() and np.all(s2[N:] == 1)
 
 
 # ------------------------------------------------------------------ cluster-segmented integer GEMM
