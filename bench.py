@@ -130,7 +130,7 @@ def _step(sites, binding, M, events=None):
 
 def run_ours(args):
     import torch
-    from paper_2304_01089_b200 import binding, workloads
+    from paper_2304_01089_b200 import binding, shard, workloads
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -197,10 +197,7 @@ def run_ours(args):
     sync_all()
     e2e_ms = e0.elapsed_time(e1)
 
-    times = torch.tensor([ms, e2e_ms], dtype=torch.float64, device="cuda")
-    if dist is not None:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    ms, e2e_ms = float(times[0]), float(times[1])
+    ms, e2e_ms = shard.max_over_ranks([ms, e2e_ms], dist, device="cuda")
 
     if rank == 0:
         peaks = _peaks()
@@ -213,7 +210,7 @@ def run_ours(args):
         ln_gbs = ln_bytes / (float(np.mean(ln_ms[1])) * 1e-3) / 1e9
         out = {
             "metric": "LN+reorder+quant GB/s and cluster W4A4 GEMM TOPS (% roofline), 9216-hidden",
-            "value": world * ops_per_step * args.steps / (ms * 1e-3) / 1e12,
+            "value": shard.aggregate_throughput(ops_per_step * args.steps, world, ms) / 1e12,
             "unit": "TOPS",
             "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
             "ms_per_step": ms / args.steps,
