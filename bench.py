@@ -97,13 +97,17 @@ def _prepare_site(sw, li, n_tokens, torch, binding):
                                 workloads.kmeans_draws(sw, 0, sw.clusters), EPS)
     L = binding.Layout(cal.perm, cal.size, cal.scale, cal.zero, sw.bits)
     n_out = sw.linears[li].n_out
-    w_codes = np.empty((n_out, L.K_pad // 2), np.uint8)
+    rb = L.K_pad // 2
+    w_codes = np.zeros(binding.weight_codes_bytes(L.K_pad, n_out), np.uint8)
     s_w = np.empty(n_out, np.float32)
     wsum = np.empty((sw.clusters, n_out), np.int32)
+    # pack in blocks of 4096 output rows (a whole number of 128-row tiles, so each block's
+    # tile-major bytes are one contiguous range of the full buffer)
     for lo, blk in workloads.weight_rows(sw, li, n_out, sw.hidden, chunk=4096):
         wc, s, ws = binding.weight_pack(L, blk)
         hi = lo + blk.shape[0]
-        w_codes[lo:hi], s_w[lo:hi], wsum[:, lo:hi] = wc, s, ws
+        w_codes[lo * rb:lo * rb + wc.shape[0]] = wc
+        s_w[lo:hi], wsum[:, lo:hi] = s, ws
     x_host = torch.from_numpy(workloads.test_tokens(sw, n_tokens)).pin_memory()
     return dict(sw=sw, L=L, cal=cal, n_out=n_out, gamma_h=gamma, beta_h=beta,
                 gamma=torch.from_numpy(gamma).cuda(), beta=torch.from_numpy(beta).cuda(),
@@ -254,7 +258,7 @@ def _oracle_sample(site, rows_ln: int, rows_gemm: int):
     x = workloads.test_tokens(sw, rows_ln)
     n_out = site["n_out"]
     w_packed = site["w"].cpu().numpy() if hasattr(site["w"], "cpu") else site["w"]
-    w_codes = oracle.unpack_weights(w_packed, site["L"].K_pad)
+    w_codes = oracle.unpack_weights(w_packed, site["L"].K_pad, n_out)
     s_w = site["s_w"].cpu().numpy() if hasattr(site["s_w"], "cpu") else site["s_w"]
     wsum = site["wsum"].cpu().numpy() if hasattr(site["wsum"], "cpu") else site["wsum"]
     t0 = time.perf_counter()

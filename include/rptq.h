@@ -31,7 +31,7 @@
  * length is K_pad = max(128, roundup128(seg_off[g])). Pad positions hold activation code 0 and
  * weight code 0.
  *
- * Packed storage, format version 1 (private to this library; read it back with the *_unpack_host
+ * Packed storage, format version 2 (private to this library; read it back with the *_unpack_host
  * helpers). A row of K_pad codes takes K_pad*bits/8 bytes:
  *   8 bit  one byte per code;
  *   4 bit  32-bit little-endian word w holds codes 8w..8w+7: byte i (0..3) carries code 8w+i in
@@ -39,7 +39,11 @@
  *   3 bit  32 codes take three words; word j carries codes 8j..8j+7 of the group as in the 4-bit
  *          layout, and bit 3 of nibble t of word j carries bit j of code 24+t (nibble t = low
  *          nibble of byte t for t < 4, high nibble of byte t-4 otherwise).
- * Weight codes are signed 4-bit two's-complement nibbles in the 4-bit layout.
+ * Weight codes are signed 4-bit two's-complement nibbles in the 4-bit word layout, stored tile-major
+ * so that one staging block is one contiguous 8 KiB copy: tile (i, kb) holds output rows
+ * 128i..128i+127 and padded positions 128kb..128kb+127 as 128 rows of 64 bytes; tiles are ordered
+ * [i][kb] with kb fastest. Rows beyond N_pad in the last tile are zero. The buffer therefore has
+ * rptq_weight_codes_bytes(K_pad, N_pad) = roundup128(N_pad) * K_pad / 2 bytes.
  */
 #ifndef RPTQ_H_
 #define RPTQ_H_
@@ -62,7 +66,7 @@ enum {
 
 enum { RPTQ_OUT_F32 = 0, RPTQ_OUT_F16 = 1, RPTQ_OUT_CODES = 2 };
 enum { RPTQ_ACT_NONE = 0, RPTQ_ACT_RELU = 1 };
-enum { RPTQ_FORMAT_VERSION = 1 };
+enum { RPTQ_FORMAT_VERSION = 2 };
 
 typedef struct rptq_layout rptq_layout_t;
 
@@ -125,7 +129,7 @@ int rptq_ln_reorder_quant(const rptq_layout_t* L, const void* x, int64_t ldx, co
  *                 row where out_perm[r] < 0; no original row may appear twice. With the array that
  *                 rptq_layout_padded_index gives for the next site, the output channels come out in
  *                 that site's padded cluster order and rptq_cluster_gemm can re-quantise them in place.
- *   w_codes_host  host, N_pad rows of K_pad/2 bytes (packed signed nibbles, padded segment layout)
+ *   w_codes_host  host, rptq_weight_codes_bytes(K_pad, N_pad) bytes (tile-major packed signed nibbles)
  *   s_w           host fp32 [N_pad]
  *   wsum          host int32 [g][N_pad]: Wsum_c[r] = sum of w_q over the channels of cluster c
  * Runs on the calling thread plus OpenMP workers; touches no device.
@@ -141,8 +145,8 @@ int rptq_weight_pack(const rptq_layout_t* Lin, const float* W_host, int N, const
  * that of the weight's rows, so a following reordered site reads it without an explicit reorder).
  *   a_codes  dev, M rows of Lin.row_bytes bytes (as written by rptq_ln_reorder_quant or by this
  *            function with RPTQ_OUT_CODES)
- *   w_codes  dev, N_pad rows of Lin.K_pad/2 bytes; s_w dev fp32 [N_pad]; wsum dev int32 [g][N_pad]
- *            (as produced by rptq_weight_pack and copied to the device); N_pad = ld_w >= N
+ *   w_codes  dev, rptq_weight_codes_bytes(Lin.K_pad, N_pad) bytes; s_w dev fp32 [N_pad]; wsum dev
+ *            int32 [g][N_pad] (as produced by rptq_weight_pack and copied to the device); N_pad = ld_w >= N
  *   bias     NULL or dev fp32 [N_pad]
  *   act      RPTQ_ACT_NONE or RPTQ_ACT_RELU
  *   y_dtype  RPTQ_OUT_F32 / RPTQ_OUT_F16: y is dev [M][ldy] of that type (ldy >= N, in elements,
@@ -171,6 +175,7 @@ int rptq_cluster_gemm_debug_acc(const rptq_layout_t* Lin, const void* a_codes, i
 int rptq_codes_unpack_host(int K_pad, int bits, const void* packed_host, int64_t M, uint8_t* codes_host);
 int rptq_codes_pack_host(int K_pad, int bits, const uint8_t* codes_host, int64_t M, void* packed_host);
 int rptq_weight_unpack_host(int K_pad, const void* packed_host, int64_t N, int8_t* w_host);
+int64_t rptq_weight_codes_bytes(int K_pad, int64_t N_pad);
 
 /*
  * Kernels never spin without a limit: a wait that runs out records RPTQ_ERR_DEVICE_TIMEOUT in a

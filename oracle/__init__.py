@@ -31,6 +31,7 @@ def _arr(a, dt) -> np.ndarray:
 
 _lib.orc_segment_offsets.restype = _i32
 _lib.orc_row_bytes.restype = _i64
+_lib.orc_weight_codes_bytes.restype = _i64
 _lib.orc_cluster_gemm.restype = _i64
 _lib.orc_kmeans.restype = C.c_int
 
@@ -160,19 +161,24 @@ def unpack(packed: np.ndarray, k_pad: int, k: int) -> np.ndarray:
     return out
 
 
+def weight_codes_bytes(n_rows: int, k_pad: int) -> int:
+    return int(_lib.orc_weight_codes_bytes(_i64(n_rows), _i32(k_pad)))
+
+
 def pack_weights(w_codes: np.ndarray) -> np.ndarray:
+    """Tile-major packed weight buffer (flat uint8) of int8 codes [N][K_pad]."""
     w_codes = _arr(w_codes, np.int8)
     N, k_pad = w_codes.shape
-    out = np.empty((N, k_pad // 2), np.uint8)
+    out = np.empty(weight_codes_bytes(N, k_pad), np.uint8)
     _lib.orc_pack_weight_codes(_p(w_codes), _i64(N), _i32(k_pad), _p(out))
     return out
 
 
-def unpack_weights(packed: np.ndarray, k_pad: int) -> np.ndarray:
-    packed = _arr(packed, np.uint8)
-    N = packed.shape[0]
-    out = np.empty((N, k_pad), np.int8)
-    _lib.orc_unpack_weight_codes(_p(packed), _i64(N), _i32(k_pad), _p(out))
+def unpack_weights(packed: np.ndarray, k_pad: int, n_rows: int) -> np.ndarray:
+    packed = _arr(packed, np.uint8).reshape(-1)
+    assert packed.shape[0] >= weight_codes_bytes(n_rows, k_pad)
+    out = np.empty((n_rows, k_pad), np.int8)
+    _lib.orc_unpack_weight_codes(_p(packed), _i64(n_rows), _i32(k_pad), _p(out))
     return out
 
 

@@ -397,22 +397,34 @@ void orc_unpack_codes(const uint8_t* packed, int64_t M, int32_t K_pad, int k, ui
     }
 }
 
-/* Signed 4-bit weight codes use the 4-bit layout above with two's-complement nibbles. */
+/* Signed 4-bit weight codes use the 4-bit word layout above with two's-complement nibbles, stored
+ * tile-major (the library's documented format): tile (i, kb) = output rows 128i..128i+127, padded
+ * positions 128kb..128kb+127, as 128 rows of 64 bytes; tiles ordered [i][kb], kb fastest; rows
+ * beyond N in the last tile are zero. Buffer size: roundup128(N) * K_pad / 2 bytes. */
+int64_t orc_weight_codes_bytes(int64_t N, int32_t K_pad) { return (N + 127) / 128 * 128 * (int64_t)(K_pad / 2); }
+
+static uint8_t* weight_piece(uint8_t* base, int64_t n, int kb, int32_t K_pad)
+{
+    int64_t tile = (n / 128) * (K_pad / 128) + kb;
+    return base + tile * 8192 + (n % 128) * 64;
+}
+
 void orc_pack_weight_codes(const int8_t* w, int64_t N, int32_t K_pad, uint8_t* packed)
 {
-    int64_t rb = K_pad / 2;
-    memset(packed, 0, (size_t)(N * rb));
+    memset(packed, 0, (size_t)orc_weight_codes_bytes(N, K_pad));
     for (int64_t n = 0; n < N; ++n)
-        for (int p = 0; p < K_pad; ++p)
-            put_nibble(packed + n * rb, p / 8, p % 8, (unsigned)w[n * K_pad + p] & 0xFu);
+        for (int p = 0; p < K_pad; ++p) {
+            int q = p % 128;
+            put_nibble(weight_piece(packed, n, p / 128, K_pad), q / 8, q % 8, (unsigned)w[n * K_pad + p] & 0xFu);
+        }
 }
 
 void orc_unpack_weight_codes(const uint8_t* packed, int64_t N, int32_t K_pad, int8_t* w)
 {
-    int64_t rb = K_pad / 2;
     for (int64_t n = 0; n < N; ++n)
         for (int p = 0; p < K_pad; ++p) {
-            int v = (int)get_nibble(packed + n * rb, p / 8, p % 8);
+            int q = p % 128;
+            int v = (int)get_nibble(weight_piece((uint8_t*)packed, n, p / 128, K_pad), q / 8, q % 8);
             w[n * K_pad + p] = (int8_t)(v >= 8 ? v - 16 : v);
         }
 }

@@ -23,7 +23,7 @@ EXPORTS = (
     "rptq_layout_create", "rptq_layout_query", "rptq_layout_destroy", "rptq_ln_reorder_quant",
     "rptq_weight_pack", "rptq_cluster_gemm", "rptq_cluster_gemm_debug_acc", "rptq_codes_unpack_host",
     "rptq_codes_pack_host", "rptq_weight_unpack_host", "rptq_get_device_status", "rptq_status_string",
-    "rptq_format_version", "rptq_layout_padded_index",
+    "rptq_format_version", "rptq_layout_padded_index", "rptq_weight_codes_bytes",
 )
 
 
@@ -51,12 +51,14 @@ def _load(path: str = LIB_PATH) -> C.CDLL:
     lib.rptq_codes_unpack_host.argtypes = [i32, i32, vp, i64, vp]
     lib.rptq_codes_pack_host.argtypes = [i32, i32, vp, i64, vp]
     lib.rptq_weight_unpack_host.argtypes = [i32, vp, i64, vp]
+    lib.rptq_weight_codes_bytes.argtypes = [i32, i64]
     lib.rptq_get_device_status.argtypes = [C.POINTER(i32)]
     lib.rptq_status_string.argtypes = [i32]
     lib.rptq_status_string.restype = C.c_char_p
     for name in EXPORTS:
-        if name != "rptq_status_string":
+        if name not in ("rptq_status_string", "rptq_weight_codes_bytes"):
             getattr(lib, name).restype = i32
+    lib.rptq_weight_codes_bytes.restype = i64
     return lib
 
 
@@ -152,8 +154,8 @@ def ln_reorder_quant(layout: Layout, x, gamma, beta, eps: float, codes, y_dbg=No
 
 
 def weight_pack(layout_in: Layout, W: np.ndarray, out_perm=None, n_pad: Optional[int] = None):
-    """rptq_weight_pack on host arrays. Returns (w_codes uint8 [N_pad][K_pad/2], s_w fp32 [N_pad],
-    wsum int32 [g][N_pad])."""
+    """rptq_weight_pack on host arrays. Returns (w_codes: flat uint8 tile-major buffer of
+    weight_codes_bytes(K_pad, N_pad) bytes, s_w fp32 [N_pad], wsum int32 [g][N_pad])."""
     W = np.ascontiguousarray(W, dtype=np.float32)
     N, Cn = W.shape
     if Cn != layout_in.C:
@@ -164,7 +166,7 @@ def weight_pack(layout_in: Layout, W: np.ndarray, out_perm=None, n_pad: Optional
         n_pad = int(op.shape[0]) if n_pad == N and op.shape[0] != N else n_pad
         if op.shape[0] != n_pad:
             raise ValueError("out_perm must have one entry per output row (N_pad)")
-    w_codes = np.empty((n_pad, layout_in.K_pad // 2), np.uint8)
+    w_codes = np.empty(weight_codes_bytes(layout_in.K_pad, n_pad), np.uint8)
     s_w = np.empty(n_pad, np.float32)
     wsum = np.empty((layout_in.g, n_pad), np.int32)
     _check(_lib.rptq_weight_pack(layout_in.handle, _np_ptr(W), N, _np_ptr(op), n_pad, _np_ptr(w_codes),
@@ -208,9 +210,15 @@ def codes_pack_host(codes: np.ndarray, bits: int) -> np.ndarray:
     return out
 
 
-def weight_unpack_host(packed: np.ndarray, k_pad: int) -> np.ndarray:
-    packed = np.ascontiguousarray(packed, dtype=np.uint8)
-    N = packed.shape[0]
+def weight_codes_bytes(k_pad: int, n_pad: int) -> int:
+    return int(_lib.rptq_weight_codes_bytes(int(k_pad), int(n_pad)))
+
+
+def weight_unpack_host(packed: np.ndarray, k_pad: int, n_rows: int) -> np.ndarray:
+    packed = np.ascontiguousarray(packed, dtype=np.uint8).reshape(-1)
+    N = int(n_rows)
+    if packed.shape[0] < weight_codes_bytes(k_pad, N):
+        raise ValueError("packed weight buffer too small")
     out = np.empty((N, k_pad), np.int8)
     _check(_lib.rptq_weight_unpack_host(int(k_pad), _np_ptr(packed), N, _np_ptr(out)), "rptq_weight_unpack_host")
     return out

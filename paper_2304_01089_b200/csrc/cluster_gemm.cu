@@ -3,22 +3,28 @@
 //   acc_c[m][n] = sum_{k in segment c} X_q[m][k] * W_q[n][k]        int32, tcgen05.mma kind::i8
 //   y[m][n]     = s_w[n] * sum_c s_c * (acc_c[m][n] - z_c * Wsum_c[n])  (+ bias) (ReLU) (re-quantise)
 //
-// One persistent CTA per SM works on 128 (tokens) x 256 (output channels) tiles. Warp roles:
-//   warp 0      TMA producer: packed activation codes [128 rows x 128 codes] and packed 4-bit
-//               weights [256 rows x 128 codes] per K block into a ring of shared-memory stages
+// Two variants of one kernel template. NCTA = 1: one persistent CTA per SM works on 128 (tokens) x
+// 256 (output channels) tiles. NCTA = 2: the two CTAs of a cluster (an SM pair) share a 256 x 256
+// tile through tcgen05.mma.cta_group::2 -- each CTA stages and unpacks its own 128 token rows and
+// its own 128 of the 256 weight rows, which halves the weight unpacking and the shared-memory
+// traffic per MMA; the first CTA of the pair issues the MMAs for both and its commits arrive on
+// both CTAs' barriers; every CTA drains its own 128 accumulator lanes. No load is multicast.
+// Warp roles (per CTA):
+//   warp 0      bulk-copy producer: one contiguous 8 KiB cp.async.bulk per 128 weight rows per K
+//               block (the packed weights are stored tile-major for this) into a ring of stages
 //   warps 4-7   unpack: packed codes -> 8-bit operands, written in the K-major 128-byte-swizzled
-//               layout that the tensor core reads (weights become 16 * w, see unpack.cuh)
-//   warp 1      MMA issuer: four 128x256x32 tcgen05.mma per K block; each cluster segment
+//               layout that the tensor core reads (weights become 16 * w, see unpack.cuh). The
+//               activation codes of a K block are 48/64/128 bytes per token row, too narrow for the
+//               copy engine to move at speed (measured: ~10 clk per row), so these warps read them
+//               straight from global memory into registers, one K block ahead
+//   warp 1      MMA issuer: four tcgen05.mma (K = 32 each) per K block; each cluster segment
 //               accumulates into one of two 256-column TMEM buffers and is committed when it ends
 //   warps 8-15  epilogue: drain a finished cluster's accumulator (tcgen05.ld), add s_c * acc into
 //               fp32 running sums held in registers while the next cluster's MMAs run; after the
 //               last cluster apply the zero-point correction, s_w, bias, activation, and store
 // Every wait is bounded: a wait that runs out sets RPTQ_ERR_DEVICE_TIMEOUT in the status word and
 // all roles drain and return.
-#include <cuda.h>
 #include <cuda_fp16.h>
-
-#include <mutex>
 
 #include "pack.cuh"
 #include "rptq_internal.h"
@@ -27,28 +33,28 @@
 namespace rptq {
 namespace gemm {
 
-constexpr int TILE_M = 128, TILE_N = 256, KBLK = 128;
-constexpr int N_P = 3;            // packed stages
-constexpr int N_U = 2;            // unpacked (operand) stages
+constexpr int TILE_M = 128, TILE_N = 256, KBLK = 128;   // TILE_M is per CTA
 constexpr int THREADS = 512;
 constexpr int UNPACK_WARP0 = 4, N_UNPACK_WARPS = 4;
 constexpr int EPI_WARP0 = 8, N_EPI_WARPS = 8;
-constexpr int A8_BYTES = TILE_M * KBLK, W8_BYTES = TILE_N * KBLK;     // 16 KB, 32 KB
-constexpr int WP_BYTES = TILE_N * KBLK / 2;                           // 16 KB packed weights per stage
+constexpr int A8_BYTES = TILE_M * KBLK;                  // 16 KiB of 8-bit activation operands per stage
+constexpr int WTILE_BYTES = 8192;                        // one packed weight tile: 128 rows x 64 bytes
 constexpr long long WAIT_BUDGET_CYCLES = 4000000000ll;   // about two seconds at the SM clock
 
-__host__ __device__ constexpr int ap_bytes(int bits) { return TILE_M * KBLK * bits / 8; }
+__host__ __device__ constexpr int w_rows(int ncta) { return TILE_N / ncta; }           // weight rows staged per CTA
+__host__ __device__ constexpr int n_p_stages(int ncta) { return ncta == 2 ? 4 : 3; }    // packed weight stages
+__host__ __device__ constexpr int n_u_stages(int ncta) { return ncta == 2 ? 4 : 3; }    // operand stages
 
 struct SmemLayout {
     int u_stage, p_stage, off_p, off_flags, off_seg_scale, off_cl_sz, off_tab, off_bar, total;
 };
-__host__ __device__ constexpr SmemLayout smem_layout(int bits)
+__host__ __device__ constexpr SmemLayout smem_layout(int ncta)
 {
     SmemLayout s{};
-    s.u_stage = A8_BYTES + W8_BYTES;
-    s.p_stage = ap_bytes(bits) + WP_BYTES;
-    s.off_p = N_U * s.u_stage;
-    s.off_flags = s.off_p + N_P * s.p_stage;
+    s.u_stage = A8_BYTES + w_rows(ncta) * KBLK;
+    s.p_stage = w_rows(ncta) * KBLK / 2;
+    s.off_p = n_u_stages(ncta) * s.u_stage;
+    s.off_flags = s.off_p + n_p_stages(ncta) * s.p_stage;
     s.off_seg_scale = s.off_flags + 2048;
     s.off_cl_sz = s.off_seg_scale + kMaxGemmSegments * 4;
     s.off_tab = s.off_cl_sz + kMaxGemmSegments * 4;
@@ -60,6 +66,10 @@ __host__ __device__ constexpr SmemLayout smem_layout(int bits)
 struct Params {
     int M, N, n_kb, n_seg, g;
     int tiles_m, n_tiles;
+    const uint8_t* a_codes;      // [M][a_row_bytes]
+    int64_t a_row_bytes;
+    const uint8_t* w_codes;      // tile-major: n_wtiles * n_kb tiles of 8 KiB
+    int n_wtiles;
     const uint8_t* step_flags;
     const float* seg_scale;
     const float* cl_sz;
@@ -87,6 +97,15 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+// Arrive on the barrier at the same shared-memory offset in CTA `rank` of the cluster.
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t bar, uint32_t rank)
+{
+    asm volatile(
+        "{\n\t.reg .b32 ra;\n\t"
+        "mapa.shared::cluster.u32 ra, %0, %1;\n\t"
+        "mbarrier.arrive.release.cluster.shared::cluster.b64 _, [ra];\n\t}"
+        ::"r"(bar), "r"(rank) : "memory");
+}
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
@@ -101,47 +120,98 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
+// The same poll with acquire semantics at cluster scope: for barriers that the other CTA of the
+// pair arrives on.
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
 // Bounded wait. Returns false when the budget ran out or another role already gave up. The common
 // case (the phase has already completed, or completes within a few polls) touches no timer; the
 // budget is counted on the SM's cycle counter, read once per batch of polls.
-__device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, bool heed_abort)
+template <bool CLUSTER_SCOPE = false>
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, bool heed_abort = true)
 {
+    auto poll = [&]() { return CLUSTER_SCOPE ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity); };
+    if (poll()) return true;
+    if (poll()) return true;
     const long long t0 = clock64();
 #pragma unroll 1
     while (true) {
 #pragma unroll 1
         for (int i = 0; i < 1024; ++i)
-            if (mbar_try_wait(bar, parity)) return true;
+            if (poll()) return true;
         if (heed_abort && *abort_flag) return false;
         if (clock64() - t0 > WAIT_BUDGET_CYCLES) { *abort_flag = 1; return false; }
     }
 }
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, bool heed_abort = true)
+__device__ __forceinline__ uint32_t cluster_ctarank()
 {
-    if (mbar_try_wait(bar, parity)) return true;
-    if (mbar_try_wait(bar, parity)) return true;
-    return mbar_wait_slow(bar, parity, abort_flag, heed_abort);
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
 }
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar)
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// One contiguous global -> shared copy by the copy engine; completion is counted on `bar`.
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar)
 {
     asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t ldg32(const void* p)
+{
+    uint32_t v;
+    asm volatile("ld.global.nc.b32 %0, [%1];" : "=r"(v) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ uint4 ldg128(const void* p)
+{
+    uint4 v;
+    asm volatile("ld.global.nc.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
 }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+template <int NCTA>
 __device__ __forceinline__ void tc_commit(uint32_t bar)
 {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    if constexpr (NCTA == 1) {
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    } else {
+        // arrives on the barrier at this offset in both CTAs of the pair
+        const uint16_t mask = 3;
+        asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                     ::"r"(bar), "h"(mask) : "memory");
+    }
 }
+template <int NCTA>
 __device__ __forceinline__ void tc_mma_i8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
 {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+    if constexpr (NCTA == 1) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+    } else {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+    }
 }
 __device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&v)[16])
 {
@@ -166,8 +236,11 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr)
     return d;
 }
 // kind::i8, D = s32, A = unsigned 8-bit (activation codes), B = signed 8-bit (weights), both
-// K-major, M = 128, N = 256.
-constexpr uint32_t kInstrDesc = (2u << 4) | (0u << 7) | (1u << 10) | ((uint32_t)(TILE_N >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
+// K-major, M = 128 per CTA, N = 256.
+__host__ __device__ constexpr uint32_t instr_desc(int ncta)
+{
+    return (2u << 4) | (0u << 7) | (1u << 10) | ((uint32_t)(TILE_N >> 3) << 17) | ((uint32_t)((TILE_M * ncta) >> 4) << 24);
+}
 
 __device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
 {
@@ -179,21 +252,18 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr)
     asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
     return v;
 }
-__device__ __forceinline__ uint32_t lds32(uint32_t addr)
-{
-    uint32_t v;
-    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
-    return v;
-}
 
-template <int BITS>
+template <int BITS, int NCTA>
 __global__ void __launch_bounds__(THREADS, 1)
-cluster_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w, const Params p)
+cluster_gemm_kernel(const Params p)
 {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
-    constexpr SmemLayout SL = smem_layout(BITS);
-    constexpr int AP_BYTES = ap_bytes(BITS);
+    constexpr SmemLayout SL = smem_layout(NCTA);
+    constexpr int W_ROWS = w_rows(NCTA);                 // weight rows this CTA stages and unpacks
+    constexpr int N_P = n_p_stages(NCTA), N_U = n_u_stages(NCTA);
+    constexpr uint32_t kInstrDesc = instr_desc(NCTA);
     // dynamic shared memory is only guaranteed 16-byte alignment: round up to the swizzle span
+    // (the offset is the same in both CTAs of a pair, as cta_group::2 descriptors require)
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem = smem_raw + (smem_base - smem_u32(smem_raw));
 
@@ -214,12 +284,16 @@ cluster_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n_steps = p.n_kb * 4;
+    const uint32_t cta_rank = NCTA == 2 ? cluster_ctarank() : 0u;       // rank 0 issues the MMAs
+    const int pair_id = (int)blockIdx.x / NCTA, n_pairs = (int)gridDim.x / NCTA;
+    // arrive on a barrier that lives in the issuing CTA of the pair
+    auto arrive_leader = [&](uint32_t b) { if constexpr (NCTA == 1) mbar_arrive(b); else mbar_arrive_remote(b, 0); };
 
     if (tid == 0) {
         for (int i = 0; i < N_P; ++i) { mbar_init(bar(B_PFULL + i), 1); mbar_init(bar(B_PEMPTY + i), N_UNPACK_WARPS); }
-        for (int i = 0; i < N_U; ++i) { mbar_init(bar(B_UFULL + i), N_UNPACK_WARPS); mbar_init(bar(B_UEMPTY + i), 1); }
+        for (int i = 0; i < N_U; ++i) { mbar_init(bar(B_UFULL + i), N_UNPACK_WARPS * NCTA); mbar_init(bar(B_UEMPTY + i), 1); }
         for (int i = 0; i < 2; ++i) {
-            mbar_init(bar(B_ACCFULL + i), 1); mbar_init(bar(B_ACCEMPTY + i), N_EPI_WARPS); mbar_init(bar(B_TAB + i), N_EPI_WARPS);
+            mbar_init(bar(B_ACCFULL + i), 1); mbar_init(bar(B_ACCEMPTY + i), N_EPI_WARPS * NCTA); mbar_init(bar(B_TAB + i), N_EPI_WARPS);
         }
         mbar_init(bar(B_DRAIN), 1);
         *s_abort = 0;
@@ -229,34 +303,44 @@ cluster_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
     for (int i = tid; i < p.n_seg; i += THREADS) s_seg_scale[i] = p.seg_scale[i] * 0.0625f;   // operands were 16 * w
     for (int i = tid; i < p.g; i += THREADS) s_cl_sz[i] = p.cl_sz[i];
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(s_tmem_ptr)) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        if constexpr (NCTA == 1) {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(s_tmem_ptr)) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(s_tmem_ptr)) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        }
     }
     tc_fence_before();
     __syncthreads();
+    if constexpr (NCTA == 2) cluster_sync_all();       // the peer's barriers exist before anything arrives on them
     tc_fence_after();
     const uint32_t tmem_base = *s_tmem_ptr;
-
 
     // The register file is re-partitioned by warpgroup (the epilogue holds 128 running sums per
     // thread); each setmaxnreg is executed by the four warps of its group at one place.
     if (warp < UNPACK_WARP0) {
       asm volatile("setmaxnreg.dec.sync.aligned.u32 24;");
       if (warp == 0) {
-        // ------------------------------------------------------------ TMA producer
+        // ------------------------------------------------------------ bulk-copy producer
         if (lane == 0) {
             uint32_t n_issued = 0;
             bool ok = true;
-            for (int t = blockIdx.x; t < p.n_tiles && ok; t += gridDim.x) {
-                const int m0 = (t % p.tiles_m) * TILE_M, n0 = (t / p.tiles_m) * TILE_N;
+            for (int t = pair_id; t < p.n_tiles && ok; t += n_pairs) {
+                // 128-row weight tiles this CTA stages; tiles past the end of the buffer are skipped
+                // (their columns are never stored)
+                const int wt0 = ((t / p.tiles_m) * TILE_N + (int)cta_rank * W_ROWS) >> 7;
+                int n_valid = p.n_wtiles - wt0;
+                n_valid = n_valid < 0 ? 0 : (n_valid > W_ROWS / 128 ? W_ROWS / 128 : n_valid);
                 for (int kb = 0; kb < p.n_kb; ++kb, ++n_issued) {
                     const int s = n_issued % N_P;
                     const uint32_t ph = (n_issued / N_P) & 1;
                     if (!mbar_wait(bar(B_PEMPTY + s), ph ^ 1, s_abort)) { ok = false; break; }
                     const uint32_t dst = smem_base + SL.off_p + s * SL.p_stage;
-                    mbar_arrive_expect_tx(bar(B_PFULL + s), AP_BYTES + WP_BYTES);
-                    tma_load_2d(dst, &tm_a, kb * (KBLK * BITS / 8), m0, bar(B_PFULL + s));
-                    tma_load_2d(dst + AP_BYTES, &tm_w, kb * (KBLK / 2), n0, bar(B_PFULL + s));
+                    mbar_arrive_expect_tx(bar(B_PFULL + s), (uint32_t)(n_valid * WTILE_BYTES));
+                    for (int j = 0; j < n_valid; ++j)
+                        bulk_load(dst + j * WTILE_BYTES, p.w_codes + ((int64_t)(wt0 + j) * p.n_kb + kb) * WTILE_BYTES,
+                                  (uint32_t)WTILE_BYTES, bar(B_PFULL + s));
                 }
             }
             if (!ok) {
@@ -266,8 +350,8 @@ cluster_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
             }
         }
       } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        // ------------------------------------------------------------ MMA issuer (first CTA of a pair only)
+        if (lane == 0 && cta_rank == 0) {
             // This lane is a single thread of dependent instructions, so the loop is kept short:
             // stage descriptors are built once, a K block's four step flags come as one word, and a
             // block that lies inside one cluster issues its four MMAs without any test.
@@ -276,41 +360,41 @@ cluster_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
             const uint64_t a_desc0 = smem_desc_sw128(smem_base), w_desc0 = smem_desc_sw128(smem_base + A8_BYTES);
             const uint32_t* flags4 = reinterpret_cast<const uint32_t*>(s_flags);
             uint32_t d_tmem = tmem_base;
-            for (int t = blockIdx.x; t < p.n_tiles && ok; t += gridDim.x) {
+            for (int t = pair_id; t < p.n_tiles && ok; t += n_pairs) {
                 for (int kb = 0; kb < p.n_kb && ok; ++kb, ++n_kb_done) {
                     const int s = n_kb_done % N_U;
-                    if (!mbar_wait(bar(B_UFULL + s), (n_kb_done / N_U) & 1, s_abort)) { ok = false; break; }
+                    if (!mbar_wait<NCTA == 2>(bar(B_UFULL + s), (n_kb_done / N_U) & 1, s_abort)) { ok = false; break; }
                     tc_fence_after();
                     // the start-address field counts 16-byte units: one stage further, 32 bytes per step
                     const uint64_t ad = a_desc0 + (uint64_t)(s * (SL.u_stage >> 4)), wd = w_desc0 + (uint64_t)(s * (SL.u_stage >> 4));
                     const uint32_t f4 = flags4[kb];
                     if (f4 == 0) {
-                        tc_mma_i8(d_tmem, ad, wd, kInstrDesc, 1u);
-                        tc_mma_i8(d_tmem, ad + 2, wd + 2, kInstrDesc, 1u);
-                        tc_mma_i8(d_tmem, ad + 4, wd + 4, kInstrDesc, 1u);
-                        tc_mma_i8(d_tmem, ad + 6, wd + 6, kInstrDesc, 1u);
+                        tc_mma_i8<NCTA>(d_tmem, ad, wd, kInstrDesc, 1u);
+                        tc_mma_i8<NCTA>(d_tmem, ad + 2, wd + 2, kInstrDesc, 1u);
+                        tc_mma_i8<NCTA>(d_tmem, ad + 4, wd + 4, kInstrDesc, 1u);
+                        tc_mma_i8<NCTA>(d_tmem, ad + 6, wd + 6, kInstrDesc, 1u);
                     } else {
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
                             const uint32_t f = (f4 >> (8 * j)) & 0xFFu;
                             if (f & STEP_SKIP) continue;
                             if (f & STEP_FIRST) {
-                                if (!mbar_wait(bar(B_ACCEMPTY + (n_seg_done & 1)), ((n_seg_done >> 1) & 1) ^ 1, s_abort)) { ok = false; break; }
+                                if (!mbar_wait<NCTA == 2>(bar(B_ACCEMPTY + (n_seg_done & 1)), ((n_seg_done >> 1) & 1) ^ 1, s_abort)) { ok = false; break; }
                                 tc_fence_after();
                             }
-                            tc_mma_i8(d_tmem, ad + 2 * j, wd + 2 * j, kInstrDesc, (f & STEP_FIRST) ? 0u : 1u);
+                            tc_mma_i8<NCTA>(d_tmem, ad + 2 * j, wd + 2 * j, kInstrDesc, (f & STEP_FIRST) ? 0u : 1u);
                             if (f & STEP_LAST) {
-                                tc_commit(bar(B_ACCFULL + (n_seg_done & 1)));
+                                tc_commit<NCTA>(bar(B_ACCFULL + (n_seg_done & 1)));
                                 ++n_seg_done;
                                 d_tmem = tmem_base + (n_seg_done & 1) * TILE_N;
                             }
                         }
                     }
-                    tc_commit(bar(B_UEMPTY + s));      // the stage may be overwritten once these MMAs have read it
+                    tc_commit<NCTA>(bar(B_UEMPTY + s));      // the stage may be overwritten once these MMAs have read it
                 }
             }
             if (!ok) {
-                tc_commit(bar(B_DRAIN));
+                tc_commit<NCTA>(bar(B_DRAIN));
                 mbar_wait(bar(B_DRAIN), 0, s_abort, false);
             }
         }
@@ -320,41 +404,68 @@ cluster_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
         asm volatile("setmaxnreg.dec.sync.aligned.u32 88;");
         const int ut = tid - UNPACK_WARP0 * 32;      // 0..127
         uint32_t n_done = 0;
-        bool ok = true;
-        const int total_kb = ((p.n_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x) * p.n_kb;
-        for (int it = 0; it < total_kb; ++it, ++n_done) {
-            const int sp = n_done % N_P, su = n_done % N_U;
-            if (!mbar_wait(bar(B_PFULL + sp), (n_done / N_P) & 1, s_abort)) { ok = false; break; }
-            if (!mbar_wait(bar(B_UEMPTY + su), ((n_done / N_U) & 1) ^ 1, s_abort)) { ok = false; break; }
-            tc_fence_after();
-            const uint32_t pa = smem_base + SL.off_p + sp * SL.p_stage, pw = pa + AP_BYTES;
-            const uint32_t a_tile = smem_base + su * SL.u_stage, w_tile = a_tile + A8_BYTES;
-            // All packed words of my 12 items first (independent loads), then unpack and store.
-            // Item i of this thread is row (ut >> 2) + 32 i, unit ut & 3, so its two chunk positions
-            // in the swizzled row are the same for every i.
-            uint32_t pa_w[4][BITS], pw_w[8][4];
+        const int total_kb = ((p.n_tiles - pair_id + n_pairs - 1) / n_pairs) * p.n_kb;
+        // Item i of this thread is row (ut >> 2) + 32 i, unit ut & 3, so its two chunk positions in
+        // the swizzled row (16-byte chunk j of row r lives at position j ^ (r & 7)) are the same for every i.
+        const int row0 = ut >> 2, unit = ut & 3, sw = row0 & 7;
+        const uint32_t off0 = row0 * 128 + (((2 * unit) ^ sw) << 4), off1 = row0 * 128 + (((2 * unit + 1) ^ sw) << 4);
+        constexpr int W_ITEMS = W_ROWS * 4 / 128;    // weight items per thread
+        // Activation codes come straight from global memory: my four items of a K block are BITS
+        // words each, at rows m0 + row0 + 32 i, byte offset kb * 16 BITS + unit * 4 BITS of the row.
+        constexpr bool PREFETCH_A = BITS <= 4;       // one K block ahead when the registers allow it
+        auto load_a = [&](int t, int kb, uint32_t (&dst)[4][BITS]) {
+            const int m0 = (t % p.tiles_m) * (TILE_M * NCTA) + (int)cta_rank * TILE_M;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                const int item = ut + i * 128;
-                if constexpr (BITS == 4) {
-                    const uint4 v = lds128(pa + item * 16);
-                    pa_w[i][0] = v.x; pa_w[i][1] = v.y; pa_w[i][2] = v.z; pa_w[i][3] = v.w;
-                } else if constexpr (BITS == 3) {
+                const int row = m0 + row0 + 32 * i;
+                const uint8_t* src = p.a_codes + (int64_t)row * p.a_row_bytes + kb * (16 * BITS) + unit * (4 * BITS);
+                if (row < p.M) {
+                    if constexpr (BITS == 3) {
 #pragma unroll
-                    for (int j = 0; j < 3; ++j) pa_w[i][j] = lds32(pa + item * 12 + j * 4);
+                        for (int j = 0; j < 3; ++j) dst[i][j] = ldg32(src + 4 * j);
+                    } else if constexpr (BITS == 4) {
+                        const uint4 v = ldg128(src);
+                        dst[i][0] = v.x; dst[i][1] = v.y; dst[i][2] = v.z; dst[i][3] = v.w;
+                    } else {
+                        const uint4 v0 = ldg128(src), v1 = ldg128(src + 16);
+                        dst[i][0] = v0.x; dst[i][1] = v0.y; dst[i][2] = v0.z; dst[i][3] = v0.w;
+                        dst[i][4] = v1.x; dst[i][5] = v1.y; dst[i][6] = v1.z; dst[i][7] = v1.w;
+                    }
                 } else {
-                    const uint4 v0 = lds128(pa + item * 32), v1 = lds128(pa + item * 32 + 16);
-                    pa_w[i][0] = v0.x; pa_w[i][1] = v0.y; pa_w[i][2] = v0.z; pa_w[i][3] = v0.w;
-                    pa_w[i][4] = v1.x; pa_w[i][5] = v1.y; pa_w[i][6] = v1.z; pa_w[i][7] = v1.w;
+#pragma unroll
+                    for (int j = 0; j < BITS; ++j) dst[i][j] = 0u;
                 }
             }
+        };
+        int t_cur = pair_id, kb_cur = 0;
+        uint32_t pa_w[4][BITS], pa_next[4][BITS];
+        if (PREFETCH_A && total_kb > 0) load_a(t_cur, kb_cur, pa_next);
+        for (int it = 0; it < total_kb; ++it, ++n_done) {
+            const int sp = n_done % N_P, su = n_done % N_U;
+            int t_nxt = t_cur, kb_nxt = kb_cur + 1;
+            if (kb_nxt == p.n_kb) { kb_nxt = 0; t_nxt += n_pairs; }
+            if constexpr (PREFETCH_A) {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
+                for (int i = 0; i < 4; ++i)
+#pragma unroll
+                    for (int j = 0; j < BITS; ++j) pa_w[i][j] = pa_next[i][j];
+                if (it + 1 < total_kb) load_a(t_nxt, kb_nxt, pa_next);
+            } else {
+                load_a(t_cur, kb_cur, pa_w);
+            }
+            t_cur = t_nxt; kb_cur = kb_nxt;
+            if (!mbar_wait(bar(B_PFULL + sp), (n_done / N_P) & 1, s_abort)) break;
+            if (!mbar_wait(bar(B_UEMPTY + su), ((n_done / N_U) & 1) ^ 1, s_abort)) break;
+            tc_fence_after();
+            const uint32_t pw = smem_base + SL.off_p + sp * SL.p_stage;
+            const uint32_t a_tile = smem_base + su * SL.u_stage, w_tile = a_tile + A8_BYTES;
+            // all packed weight words of my items first (independent loads), then unpack and store
+            uint32_t pw_w[W_ITEMS][4];
+#pragma unroll
+            for (int i = 0; i < W_ITEMS; ++i) {
                 const uint4 v = lds128(pw + (ut + i * 128) * 16);
                 pw_w[i][0] = v.x; pw_w[i][1] = v.y; pw_w[i][2] = v.z; pw_w[i][3] = v.w;
             }
-            const int row0 = ut >> 2, unit = ut & 3, sw = row0 & 7;
-            const uint32_t off0 = row0 * 128 + (((2 * unit) ^ sw) << 4), off1 = row0 * 128 + (((2 * unit + 1) ^ sw) << 4);
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 uint32_t o[8];
@@ -363,7 +474,7 @@ cluster_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
                 sts128(a_tile + off1 + i * 4096, o[4], o[5], o[6], o[7]);
             }
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
+            for (int i = 0; i < W_ITEMS; ++i) {
                 uint32_t o[8];
                 unpack_w32_x16(pw_w[i], o);
                 sts128(w_tile + off0 + i * 4096, o[0], o[1], o[2], o[3]);
@@ -371,9 +482,8 @@ cluster_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
             }
             fence_proxy_async();          // make the generic-proxy stores visible to the tensor core
             __syncwarp();
-            if (lane == 0) { mbar_arrive(bar(B_UFULL + su)); mbar_arrive(bar(B_PEMPTY + sp)); }
+            if (lane == 0) { arrive_leader(bar(B_UFULL + su)); mbar_arrive(bar(B_PEMPTY + sp)); }
         }
-        (void)ok;
     } else {
         // ------------------------------------------------------------ epilogue warps
         asm volatile("setmaxnreg.inc.sync.aligned.u32 200;");
@@ -383,8 +493,8 @@ cluster_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
         uint32_t n_seg_done = 0, n_tile_done = 0;
         bool ok = true;
         float R[128];
-        for (int t = blockIdx.x; t < p.n_tiles && ok; t += gridDim.x, ++n_tile_done) {
-            const int m0 = (t % p.tiles_m) * TILE_M, n0 = (t / p.tiles_m) * TILE_N;
+        for (int t = pair_id; t < p.n_tiles && ok; t += n_pairs, ++n_tile_done) {
+            const int m0 = (t % p.tiles_m) * (TILE_M * NCTA) + (int)cta_rank * TILE_M, n0 = (t / p.tiles_m) * TILE_N;
             float* tab = s_tab + (n_tile_done & 1) * 3 * TILE_N;
             {   // per-tile column constants: zero-point correction sum_c s_c z_c Wsum_c[n], s_w[n], bias[n]
                 const int n = n0 + et;
@@ -421,7 +531,7 @@ cluster_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
                 }
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(B_ACCEMPTY + buf));
+                if (lane == 0) arrive_leader(bar(B_ACCEMPTY + buf));
             }
             if (!ok) break;
             if (!mbar_wait(bar(B_TAB + (n_tile_done & 1)), (n_tile_done >> 1) & 1, s_abort)) { ok = false; break; }
@@ -498,60 +608,40 @@ cluster_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
     // ---------------------------------------------------------------- teardown
     tc_fence_before();
     __syncthreads();
+    if constexpr (NCTA == 2) cluster_sync_all();       // the peer no longer arrives here nor reads this CTA's memory
     tc_fence_after();
     if (warp == 1) {
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
+        if constexpr (NCTA == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
+        else asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
     }
     if (tid == 0 && *s_abort && p.status) atomicExch(p.status, RPTQ_ERR_DEVICE_TIMEOUT);
 }
 
 // ---------------------------------------------------------------- host side
-using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                              const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeFn encode_fn()
+template <int BITS, int NCTA>
+static int launch(const Params& p, int n_sm, cudaStream_t st)
 {
-    static std::once_flag once;
-    static EncodeFn fn = nullptr;
-    std::call_once(once, [] {
-        void* sym = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeFn>(sym);
-    });
-    return fn;
-}
-
-// 2-D byte tensor [rows][row_bytes], box [box_rows][box_bytes], no swizzle, zero fill out of range.
-static int make_map(CUtensorMap* map, const void* base, uint64_t row_bytes, uint64_t rows, uint32_t box_bytes, uint32_t box_rows)
-{
-    EncodeFn fn = encode_fn();
-    if (!fn) return RPTQ_ERR_CUDA;
-    const cuuint64_t dims[2] = {row_bytes, rows};
-    const cuuint64_t strides[1] = {row_bytes};
-    const cuuint32_t box[2] = {box_bytes, box_rows};
-    const cuuint32_t estr[2] = {1, 1};
-    const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
-                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS ? RPTQ_OK : RPTQ_ERR_CUDA;
-}
-
-template <int BITS>
-static int launch(const CUtensorMap& tm_a, const CUtensorMap& tm_w, const Params& p, int grid, cudaStream_t st)
-{
-    constexpr SmemLayout SL = smem_layout(BITS);
+    constexpr SmemLayout SL = smem_layout(NCTA);
     const int smem = SL.total + 1024;     // slack for the in-kernel 1024-byte alignment
-    const void* fn = reinterpret_cast<const void*>(cluster_gemm_kernel<BITS>);
+    const void* fn = reinterpret_cast<const void*>(cluster_gemm_kernel<BITS, NCTA>);
     cudaFuncAttributes attr;
     if (cudaFuncGetAttributes(&attr, fn) != cudaSuccess) return RPTQ_ERR_CUDA;
     // the register re-partition inside the kernel (setmaxnreg) assumes this pool; refuse to launch otherwise
     if (attr.numRegs * THREADS < 24 * 128 + 88 * 128 + 200 * 256) return RPTQ_ERR_UNSUPPORTED;
     if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return RPTQ_ERR_CUDA;
-    cluster_gemm_kernel<BITS><<<grid, THREADS, smem, st>>>(tm_a, tm_w, p);
-    return cudaGetLastError() == cudaSuccess ? RPTQ_OK : RPTQ_ERR_CUDA;
+    const int slots = n_sm / NCTA;
+    const int groups = p.n_tiles < slots ? p.n_tiles : slots;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)(groups * NCTA));
+    cfg.blockDim = dim3(THREADS);
+    cfg.dynamicSmemBytes = (size_t)smem;
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = NCTA; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, cluster_gemm_kernel<BITS, NCTA>, p) == cudaSuccess ? RPTQ_OK : RPTQ_ERR_CUDA;
 }
 
 }  // namespace gemm
@@ -585,8 +675,12 @@ extern "C" int rptq_cluster_gemm(const rptq_layout_t* Lin, const void* a_codes, 
 
     gemm::Params p{};
     p.M = M; p.N = N; p.n_kb = Lin->K_pad / gemm::KBLK; p.n_seg = Lin->n_seg; p.g = Lin->g;
-    p.tiles_m = (M + gemm::TILE_M - 1) / gemm::TILE_M;
+    // CTA pairs share a 256-row tile; one token tile or less gains nothing from pairing
+    const int ncta = M > gemm::TILE_M ? 2 : 1;
+    p.tiles_m = (M + gemm::TILE_M * ncta - 1) / (gemm::TILE_M * ncta);
     p.n_tiles = p.tiles_m * ((N + gemm::TILE_N - 1) / gemm::TILE_N);
+    p.a_codes = static_cast<const uint8_t*>(a_codes); p.a_row_bytes = Lin->row_bytes;
+    p.w_codes = static_cast<const uint8_t*>(w_codes); p.n_wtiles = (int)((ld_w + 127) / 128);
     p.step_flags = Lin->d_step_flags; p.seg_scale = Lin->d_seg_scale; p.cl_sz = Lin->d_cl_sz;
     p.s_w = s_w; p.wsum = wsum; p.ld_w = ld_w; p.bias = static_cast<const float*>(bias);
     p.act = act; p.y_dtype = y_dtype; p.y = y; p.ldy = ldy;
@@ -596,17 +690,15 @@ extern "C" int rptq_cluster_gemm(const rptq_layout_t* Lin, const void* a_codes, 
     p.status = device_status_word();
     if (!p.status) return RPTQ_ERR_ALLOC;
 
-    CUtensorMap tm_a, tm_w;
-    int rc = gemm::make_map(&tm_a, a_codes, (uint64_t)Lin->row_bytes, (uint64_t)M, (uint32_t)(gemm::KBLK * Lin->bits / 8), gemm::TILE_M);
-    if (rc != RPTQ_OK) return rc;
-    rc = gemm::make_map(&tm_w, w_codes, (uint64_t)Lin->K_pad / 2, (uint64_t)ld_w, gemm::KBLK / 2, gemm::TILE_N);
-    if (rc != RPTQ_OK) return rc;
-
     int n_sm = 0;
     if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return RPTQ_ERR_CUDA;
-    const int grid = p.n_tiles < n_sm ? p.n_tiles : n_sm;
     auto st = static_cast<cudaStream_t>(stream);
-    if (Lin->bits == 3) return gemm::launch<3>(tm_a, tm_w, p, grid, st);
-    if (Lin->bits == 4) return gemm::launch<4>(tm_a, tm_w, p, grid, st);
-    return gemm::launch<8>(tm_a, tm_w, p, grid, st);
+    if (ncta == 2) {
+        if (Lin->bits == 3) return gemm::launch<3, 2>(p, n_sm, st);
+        if (Lin->bits == 4) return gemm::launch<4, 2>(p, n_sm, st);
+        return gemm::launch<8, 2>(p, n_sm, st);
+    }
+    if (Lin->bits == 3) return gemm::launch<3, 1>(p, n_sm, st);
+    if (Lin->bits == 4) return gemm::launch<4, 1>(p, n_sm, st);
+    return gemm::launch<8, 1>(p, n_sm, st);
 }

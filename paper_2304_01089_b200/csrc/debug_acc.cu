@@ -16,7 +16,7 @@ __device__ __forceinline__ int dp4a_u8_s8(uint32_t a, uint32_t b, int c)
 
 template <int BITS>
 __global__ void debug_acc_kernel(const uint8_t* __restrict__ a_codes, int64_t a_row_bytes,
-                                 const uint8_t* __restrict__ w_codes, int64_t w_row_bytes,
+                                 const uint8_t* __restrict__ w_codes, int n_kb,
                                  const int32_t* __restrict__ seg_off, int g, int m0, int m1, int n0, int n1,
                                  int32_t* __restrict__ acc)
 {
@@ -26,14 +26,13 @@ __global__ void debug_acc_kernel(const uint8_t* __restrict__ a_codes, int64_t a_
     if (n >= n1 || m >= m1) return;
     const int step_lo = seg_off[c] / 32, step_hi = (seg_off[c + 1]) / 32;
     const uint32_t* arow = reinterpret_cast<const uint32_t*>(a_codes + (int64_t)m * a_row_bytes);
-    const uint32_t* wrow = reinterpret_cast<const uint32_t*>(w_codes + (int64_t)n * w_row_bytes);
     int sum = 0;
     for (int s = step_lo; s < step_hi; ++s) {
         uint32_t ap[BITS], wp[4], a8[8], w8[8];
 #pragma unroll
         for (int i = 0; i < BITS; ++i) ap[i] = arow[s * BITS + i];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) wp[i] = wrow[s * 4 + i];
+        for (int i = 0; i < 4; ++i) wp[i] = reinterpret_cast<const uint32_t*>(w_codes + weight_tile_offset(n, s >> 2, n_kb) + (s & 3) * 16)[i];
         unpack_act32<BITS>(ap, a8);
         unpack_w32_x16(wp, w8);
 #pragma unroll
@@ -62,7 +61,7 @@ extern "C" int rptq_cluster_gemm_debug_acc(const rptq_layout_t* Lin, const void*
     auto st = static_cast<cudaStream_t>(stream);
     const auto* a = static_cast<const uint8_t*>(a_codes);
     const auto* w = static_cast<const uint8_t*>(w_codes);
-    const int64_t wrb = Lin->K_pad / 2;
+    const int wrb = Lin->K_pad / 128;      // K blocks per row of the tile-major weight buffer
     if (Lin->bits == 3) debug_acc_kernel<3><<<grid, block, 0, st>>>(a, Lin->row_bytes, w, wrb, Lin->d_seg_off, Lin->g, m0, m1, n0, n1, acc);
     else if (Lin->bits == 4) debug_acc_kernel<4><<<grid, block, 0, st>>>(a, Lin->row_bytes, w, wrb, Lin->d_seg_off, Lin->g, m0, m1, n0, n1, acc);
     else debug_acc_kernel<8><<<grid, block, 0, st>>>(a, Lin->row_bytes, w, wrb, Lin->d_seg_off, Lin->g, m0, m1, n0, n1, acc);

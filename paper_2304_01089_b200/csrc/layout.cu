@@ -254,13 +254,20 @@ int rptq_codes_unpack_host(int K_pad, int bits, const void* packed_host, int64_t
     return RPTQ_OK;
 }
 
+int64_t rptq_weight_codes_bytes(int K_pad, int64_t N_pad)
+{
+    if (K_pad <= 0 || K_pad % 128 || N_pad < 0) return RPTQ_ERR_INVALID_ARG;
+    return (N_pad + 127) / 128 * 128 * (int64_t)(K_pad / 2);
+}
+
 int rptq_weight_unpack_host(int K_pad, const void* packed_host, int64_t N, int8_t* w_host)
 {
     if (!w_host || !packed_host || N < 0 || K_pad <= 0 || K_pad % 128) return RPTQ_ERR_INVALID_ARG;
-    const int64_t rb = K_pad / 2;
+    const int n_kb = K_pad / 128;
     for (int64_t n = 0; n < N; ++n) {
         uint8_t* dst = reinterpret_cast<uint8_t*>(w_host) + n * K_pad;
-        unpack_row(static_cast<const uint8_t*>(packed_host) + n * rb, K_pad, 4, dst);
+        for (int kb = 0; kb < n_kb; ++kb)     // one 64-byte piece of the row per tile
+            unpack_row(static_cast<const uint8_t*>(packed_host) + weight_tile_offset(n, kb, n_kb), 128, 4, dst + 128 * kb);
         for (int p = 0; p < K_pad; ++p) dst[p] = (uint8_t)((dst[p] ^ 8u) - 8u);   // sign-extend the nibble
     }
     return RPTQ_OK;
@@ -280,14 +287,19 @@ int rptq_weight_pack(const rptq_layout_t* Lin, const float* W_host, int N, const
             seen[out_perm[r]] = 1;
         }
     }
-    const int64_t rb = K_pad / 2;
+    const int n_kb = K_pad / 128;
+    const int rows_stored = (N_pad + 127) / 128 * 128;        // the last tile is filled with zero rows
     uint8_t* packed = static_cast<uint8_t*>(w_codes_host);
     int failed = 0;
 #pragma omp parallel
     {
-        std::vector<uint8_t> row((size_t)K_pad);
+        std::vector<uint8_t> row((size_t)K_pad), row_packed((size_t)K_pad / 2);
 #pragma omp for schedule(static)
-        for (int r = 0; r < N_pad; ++r) {
+        for (int r = 0; r < rows_stored; ++r) {
+            if (r >= N_pad) {
+                for (int kb = 0; kb < n_kb; ++kb) std::memset(packed + weight_tile_offset(r, kb, n_kb), 0, 64);
+                continue;
+            }
             std::memset(row.data(), 0, (size_t)K_pad);
             float s = 1.0f;
             const int src_row = out_perm ? out_perm[r] : (r < N ? r : -1);
@@ -314,7 +326,8 @@ int rptq_weight_pack(const rptq_layout_t* Lin, const float* W_host, int N, const
                 for (int c = 0; c < g; ++c) wsum[(int64_t)c * N_pad + r] = 0;
             }
             s_w[r] = s;
-            pack_row(row.data(), K_pad, 4, packed + r * rb);
+            pack_row(row.data(), K_pad, 4, row_packed.data());
+            for (int kb = 0; kb < n_kb; ++kb) std::memcpy(packed + weight_tile_offset(r, kb, n_kb), row_packed.data() + 64 * kb, 64);
         }
     }
     return failed ? RPTQ_ERR_INVALID_ARG : RPTQ_OK;

@@ -30,6 +30,9 @@ constexpr int kMaxGemmSegments = 1024;
 // of a warp are contiguous across lanes; slot C holds the value that pad positions read.
 __host__ __device__ inline int ybuf_addr(int c, int C) { return ((c >> 3) << 2) + (c & 3) + ((c >> 2) & 1) * (C >> 1); }
 
+// Byte offset of the 64-byte piece (row n, K block kb) in the tile-major packed weight buffer.
+__host__ __device__ inline int64_t weight_tile_offset(int64_t n, int kb, int n_kb) { return ((n >> 7) * n_kb + kb) * 8192 + (n & 127) * 64; }
+
 }  // namespace rptq
 
 struct rptq_layout {

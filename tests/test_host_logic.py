@@ -31,7 +31,7 @@ def test_library_exports_every_declared_symbol(binding):
     lib = ctypes.CDLL(binding.LIB_PATH)
     for name in declared:
         assert hasattr(lib, name), name
-    assert binding.format_version() == 1
+    assert binding.format_version() == 2
     assert binding.status_string(-3) == "reorder index is not a bijection"
 
 
@@ -73,7 +73,8 @@ def test_packed_format_helpers_agree_with_the_oracle(binding, bits):
         assert np.array_equal(packed, oracle.pack(codes, bits))
         assert np.array_equal(binding.codes_unpack_host(packed, k_pad, bits), codes)
     w = rng.integers(-8, 8, size=(5, 256), dtype=np.int8)
-    assert np.array_equal(binding.weight_unpack_host(oracle.pack_weights(w), 256), w)
+    assert np.array_equal(binding.weight_unpack_host(oracle.pack_weights(w), 256, 5), w)
+    assert binding.weight_codes_bytes(256, 5) == 128 * 128 == oracle.weight_codes_bytes(5, 256)
 
 
 def test_weight_pack_matches_the_oracle_bit_for_bit(binding):

@@ -268,11 +268,19 @@ def test_weight_pack_round_trip_and_twos_complement_nibbles():
     r = _rng(75)
     w = r.integers(-8, 8, size=(6, 256), dtype=np.int8)
     packed = oracle.pack_weights(w)
-    assert np.array_equal(oracle.unpack_weights(packed, 256), w)
+    assert packed.shape == (128 * 128,)                       # 6 rows round up to one 128-row tile
+    assert np.array_equal(oracle.unpack_weights(packed, 256, 6), w)
     one = np.zeros((1, 128), np.int8)
     one[0, 0], one[0, 4], one[0, 1] = -1, -8, 7
-    p = oracle.pack_weights(one)[0]
+    p = oracle.pack_weights(one)
     assert p[0] == 0x8F and p[1] == 0x07
+    # tile-major placement, worked by hand: row 129, position 130 of K_pad = 256 lies in tile
+    # (1, 1) = tile number 1*2+1 = 3 (8192 bytes each), row 1 of the tile (64 bytes each), position 2
+    # of the block = low nibble of byte 2
+    big = np.zeros((130, 256), np.int8)
+    big[129, 130] = -3
+    pb = oracle.pack_weights(big)
+    assert pb.shape == (2 * 128 * 128,) and pb[3 * 8192 + 64 + 2] == 0x0D and pb.sum() == 0x0D
 
 
 # ------------------------------------------------------------------ weights
