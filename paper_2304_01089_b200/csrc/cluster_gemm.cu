@@ -15,8 +15,9 @@
 //   warps 4-7   unpack: packed codes -> 8-bit operands, written in the K-major 128-byte-swizzled
 //               layout that the tensor core reads (weights become 16 * w, see unpack.cuh). The
 //               activation codes of a K block are 48/64/128 bytes per token row, too narrow for the
-//               copy engine to move at speed (measured: ~10 clk per row), so these warps read them
-//               straight from global memory into registers, one K block ahead
+//               copy engine to move at speed (measured: ~10 clk per row), so each unpack thread
+//               fetches the words of its own items with cp.async into a private ring of
+//               shared-memory slots, several K blocks ahead
 //   warp 1      MMA issuer: four tcgen05.mma (K = 32 each) per K block; each cluster segment
 //               accumulates into one of two 256-column TMEM buffers and is committed when it ends
 //   warps 8-15  epilogue: drain a finished cluster's accumulator (tcgen05.ld), add s_c * acc into
@@ -43,18 +44,24 @@ constexpr long long WAIT_BUDGET_CYCLES = 4000000000ll;   // about two seconds at
 
 __host__ __device__ constexpr int w_rows(int ncta) { return TILE_N / ncta; }           // weight rows staged per CTA
 __host__ __device__ constexpr int n_p_stages(int ncta) { return ncta == 2 ? 4 : 3; }    // packed weight stages
-__host__ __device__ constexpr int n_u_stages(int ncta) { return ncta == 2 ? 4 : 3; }    // operand stages
+__host__ __device__ constexpr int n_u_stages(int ncta) { return ncta == 2 ? 4 : 2; }    // operand stages
+// ring of packed activation K blocks fetched ahead by the unpack threads: 512 items per K block,
+// one 16-byte slot per item (two for 8-bit codes)
+__host__ __device__ constexpr int a_slot_bytes(int bits) { return bits == 8 ? 32 : 16; }
+__host__ __device__ constexpr int n_a_stages(int bits) { return bits == 8 ? 2 : 4; }
 
 struct SmemLayout {
-    int u_stage, p_stage, off_p, off_flags, off_seg_scale, off_cl_sz, off_tab, off_bar, total;
+    int u_stage, p_stage, a_stage, off_p, off_a, off_flags, off_seg_scale, off_cl_sz, off_tab, off_bar, total;
 };
-__host__ __device__ constexpr SmemLayout smem_layout(int ncta)
+__host__ __device__ constexpr SmemLayout smem_layout(int ncta, int bits)
 {
     SmemLayout s{};
     s.u_stage = A8_BYTES + w_rows(ncta) * KBLK;
     s.p_stage = w_rows(ncta) * KBLK / 2;
+    s.a_stage = 512 * a_slot_bytes(bits);
     s.off_p = n_u_stages(ncta) * s.u_stage;
-    s.off_flags = s.off_p + n_p_stages(ncta) * s.p_stage;
+    s.off_a = s.off_p + n_p_stages(ncta) * s.p_stage;
+    s.off_flags = s.off_a + n_a_stages(bits) * s.a_stage;
     s.off_seg_scale = s.off_flags + 2048;
     s.off_cl_sz = s.off_seg_scale + kMaxGemmSegments * 4;
     s.off_tab = s.off_cl_sz + kMaxGemmSegments * 4;
@@ -103,7 +110,7 @@ __device__ __forceinline__ void mbar_arrive_remote(uint32_t bar, uint32_t rank)
     asm volatile(
         "{\n\t.reg .b32 ra;\n\t"
         "mapa.shared::cluster.u32 ra, %0, %1;\n\t"
-        "mbarrier.arrive.release.cluster.shared::cluster.b64 _, [ra];\n\t}"
+        "mbarrier.arrive.shared::cluster.b64 _, [ra];\n\t}"
         ::"r"(bar), "r"(rank) : "memory");
 }
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
@@ -120,25 +127,12 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// The same poll with acquire semantics at cluster scope: for barriers that the other CTA of the
-// pair arrives on.
-__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
 // Bounded wait. Returns false when the budget ran out or another role already gave up. The common
 // case (the phase has already completed, or completes within a few polls) touches no timer; the
 // budget is counted on the SM's cycle counter, read once per batch of polls.
-template <bool CLUSTER_SCOPE = false>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, bool heed_abort = true)
 {
-    auto poll = [&]() { return CLUSTER_SCOPE ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity); };
+    auto poll = [&]() { return mbar_try_wait(bar, parity); };
     if (poll()) return true;
     if (poll()) return true;
     const long long t0 = clock64();
@@ -169,18 +163,21 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
         "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
         ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
-__device__ __forceinline__ uint32_t ldg32(const void* p)
+// Asynchronous global -> shared copies of 4 or 16 bytes issued by ordinary threads; `valid` false
+// writes zeros and reads nothing.
+__device__ __forceinline__ void cp_async4(uint32_t dst, const void* src, bool valid)
 {
-    uint32_t v;
-    asm volatile("ld.global.nc.b32 %0, [%1];" : "=r"(v) : "l"(p));
-    return v;
+    const uint32_t n = valid ? 4u : 0u;
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(n) : "memory");
 }
-__device__ __forceinline__ uint4 ldg128(const void* p)
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool valid)
 {
-    uint4 v;
-    asm volatile("ld.global.nc.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-    return v;
+    const uint32_t n = valid ? 16u : 0u;
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(n) : "memory");
 }
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -258,7 +255,7 @@ __global__ void __launch_bounds__(THREADS, 1)
 cluster_gemm_kernel(const Params p)
 {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
-    constexpr SmemLayout SL = smem_layout(NCTA);
+    constexpr SmemLayout SL = smem_layout(NCTA, BITS);
     constexpr int W_ROWS = w_rows(NCTA);                 // weight rows this CTA stages and unpacks
     constexpr int N_P = n_p_stages(NCTA), N_U = n_u_stages(NCTA);
     constexpr uint32_t kInstrDesc = instr_desc(NCTA);
@@ -363,7 +360,7 @@ cluster_gemm_kernel(const Params p)
             for (int t = pair_id; t < p.n_tiles && ok; t += n_pairs) {
                 for (int kb = 0; kb < p.n_kb && ok; ++kb, ++n_kb_done) {
                     const int s = n_kb_done % N_U;
-                    if (!mbar_wait<NCTA == 2>(bar(B_UFULL + s), (n_kb_done / N_U) & 1, s_abort)) { ok = false; break; }
+                    if (!mbar_wait(bar(B_UFULL + s), (n_kb_done / N_U) & 1, s_abort)) { ok = false; break; }
                     tc_fence_after();
                     // the start-address field counts 16-byte units: one stage further, 32 bytes per step
                     const uint64_t ad = a_desc0 + (uint64_t)(s * (SL.u_stage >> 4)), wd = w_desc0 + (uint64_t)(s * (SL.u_stage >> 4));
@@ -379,7 +376,7 @@ cluster_gemm_kernel(const Params p)
                             const uint32_t f = (f4 >> (8 * j)) & 0xFFu;
                             if (f & STEP_SKIP) continue;
                             if (f & STEP_FIRST) {
-                                if (!mbar_wait<NCTA == 2>(bar(B_ACCEMPTY + (n_seg_done & 1)), ((n_seg_done >> 1) & 1) ^ 1, s_abort)) { ok = false; break; }
+                                if (!mbar_wait(bar(B_ACCEMPTY + (n_seg_done & 1)), ((n_seg_done >> 1) & 1) ^ 1, s_abort)) { ok = false; break; }
                                 tc_fence_after();
                             }
                             tc_mma_i8<NCTA>(d_tmem, ad + 2 * j, wd + 2 * j, kInstrDesc, (f & STEP_FIRST) ? 0u : 1u);
@@ -410,50 +407,59 @@ cluster_gemm_kernel(const Params p)
         const int row0 = ut >> 2, unit = ut & 3, sw = row0 & 7;
         const uint32_t off0 = row0 * 128 + (((2 * unit) ^ sw) << 4), off1 = row0 * 128 + (((2 * unit + 1) ^ sw) << 4);
         constexpr int W_ITEMS = W_ROWS * 4 / 128;    // weight items per thread
-        // Activation codes come straight from global memory: my four items of a K block are BITS
-        // words each, at rows m0 + row0 + 32 i, byte offset kb * 16 BITS + unit * 4 BITS of the row.
-        constexpr bool PREFETCH_A = BITS <= 4;       // one K block ahead when the registers allow it
-        auto load_a = [&](int t, int kb, uint32_t (&dst)[4][BITS]) {
+        // Activation codes: my four items of a K block are BITS words each, at rows m0 + row0 + 32 i,
+        // byte offset kb * 16 BITS + unit * 4 BITS of the row. They are fetched N_A - 1 K blocks ahead
+        // into slots that only this thread reads, so no other thread has to be waited for.
+        constexpr int N_A = n_a_stages(BITS), SLOT = a_slot_bytes(BITS);
+        const uint32_t a_ring = smem_base + SL.off_a + ut * SLOT;
+        auto fetch_a = [&](int t, int kb, int stage) {
             const int m0 = (t % p.tiles_m) * (TILE_M * NCTA) + (int)cta_rank * TILE_M;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const int row = m0 + row0 + 32 * i;
-                const uint8_t* src = p.a_codes + (int64_t)row * p.a_row_bytes + kb * (16 * BITS) + unit * (4 * BITS);
-                if (row < p.M) {
-                    if constexpr (BITS == 3) {
+                const bool valid = row < p.M;
+                const uint8_t* src = p.a_codes + (int64_t)(valid ? row : 0) * p.a_row_bytes + kb * (16 * BITS) + unit * (4 * BITS);
+                const uint32_t dst = a_ring + stage * SL.a_stage + i * 128 * SLOT;
+                if constexpr (BITS == 3) {
 #pragma unroll
-                        for (int j = 0; j < 3; ++j) dst[i][j] = ldg32(src + 4 * j);
-                    } else if constexpr (BITS == 4) {
-                        const uint4 v = ldg128(src);
-                        dst[i][0] = v.x; dst[i][1] = v.y; dst[i][2] = v.z; dst[i][3] = v.w;
-                    } else {
-                        const uint4 v0 = ldg128(src), v1 = ldg128(src + 16);
-                        dst[i][0] = v0.x; dst[i][1] = v0.y; dst[i][2] = v0.z; dst[i][3] = v0.w;
-                        dst[i][4] = v1.x; dst[i][5] = v1.y; dst[i][6] = v1.z; dst[i][7] = v1.w;
-                    }
+                    for (int j = 0; j < 3; ++j) cp_async4(dst + 4 * j, src + 4 * j, valid);
+                } else if constexpr (BITS == 4) {
+                    cp_async16(dst, src, valid);
                 } else {
-#pragma unroll
-                    for (int j = 0; j < BITS; ++j) dst[i][j] = 0u;
+                    cp_async16(dst, src, valid);
+                    cp_async16(dst + 16, src + 16, valid);
                 }
             }
         };
-        int t_cur = pair_id, kb_cur = 0;
-        uint32_t pa_w[4][BITS], pa_next[4][BITS];
-        if (PREFETCH_A && total_kb > 0) load_a(t_cur, kb_cur, pa_next);
+        int t_f = pair_id, kb_f = 0, n_fetched = 0;      // next K block to fetch
+        auto fetch_next = [&]() {
+            if (n_fetched < total_kb) {
+                fetch_a(t_f, kb_f, n_fetched % N_A);
+                if (++kb_f == p.n_kb) { kb_f = 0; t_f += n_pairs; }
+            }
+            ++n_fetched;
+            cp_async_commit();                           // one group per K block, empty past the end
+        };
+#pragma unroll 1
+        for (int i = 0; i < N_A - 1; ++i) fetch_next();
         for (int it = 0; it < total_kb; ++it, ++n_done) {
             const int sp = n_done % N_P, su = n_done % N_U;
-            int t_nxt = t_cur, kb_nxt = kb_cur + 1;
-            if (kb_nxt == p.n_kb) { kb_nxt = 0; t_nxt += n_pairs; }
-            if constexpr (PREFETCH_A) {
+            fetch_next();
+            cp_async_wait<N_A - 1>();                    // the group of K block `it` has landed
+            uint32_t pa_w[4][BITS];
+            {
+                const uint32_t slot = a_ring + (it % N_A) * SL.a_stage;
 #pragma unroll
-                for (int i = 0; i < 4; ++i)
-#pragma unroll
-                    for (int j = 0; j < BITS; ++j) pa_w[i][j] = pa_next[i][j];
-                if (it + 1 < total_kb) load_a(t_nxt, kb_nxt, pa_next);
-            } else {
-                load_a(t_cur, kb_cur, pa_w);
+                for (int i = 0; i < 4; ++i) {
+                    const uint4 v = lds128(slot + i * 128 * SLOT);
+                    if constexpr (BITS == 3) { pa_w[i][0] = v.x; pa_w[i][1] = v.y; pa_w[i][2] = v.z; }
+                    else { pa_w[i][0] = v.x; pa_w[i][1] = v.y; pa_w[i][2] = v.z; pa_w[i][3] = v.w; }
+                    if constexpr (BITS == 8) {
+                        const uint4 u = lds128(slot + i * 128 * SLOT + 16);
+                        pa_w[i][4] = u.x; pa_w[i][5] = u.y; pa_w[i][6] = u.z; pa_w[i][7] = u.w;
+                    }
+                }
             }
-            t_cur = t_nxt; kb_cur = kb_nxt;
             if (!mbar_wait(bar(B_PFULL + sp), (n_done / N_P) & 1, s_abort)) break;
             if (!mbar_wait(bar(B_UEMPTY + su), ((n_done / N_U) & 1) ^ 1, s_abort)) break;
             tc_fence_after();
@@ -621,7 +627,7 @@ cluster_gemm_kernel(const Params p)
 template <int BITS, int NCTA>
 static int launch(const Params& p, int n_sm, cudaStream_t st)
 {
-    constexpr SmemLayout SL = smem_layout(NCTA);
+    constexpr SmemLayout SL = smem_layout(NCTA, BITS);
     const int smem = SL.total + 1024;     // slack for the in-kernel 1024-byte alignment
     const void* fn = reinterpret_cast<const void*>(cluster_gemm_kernel<BITS, NCTA>);
     cudaFuncAttributes attr;
