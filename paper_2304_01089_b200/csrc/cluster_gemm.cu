@@ -45,9 +45,10 @@ constexpr long long WAIT_BUDGET_CYCLES = 4000000000ll;   // about two seconds at
 __host__ __device__ constexpr int w_rows(int ncta) { return TILE_N / ncta; }           // weight rows staged per CTA
 __host__ __device__ constexpr int n_p_stages(int ncta) { return ncta == 2 ? 4 : 3; }    // packed weight stages
 __host__ __device__ constexpr int n_u_stages(int ncta) { return ncta == 2 ? 4 : 2; }    // operand stages
-// ring of packed activation K blocks fetched ahead by the unpack threads: 512 items per K block,
-// one 16-byte slot per item (two for 8-bit codes)
-__host__ __device__ constexpr int a_slot_bytes(int bits) { return bits == 8 ? 32 : 16; }
+// ring of packed activation K blocks fetched ahead by the unpack threads: one slot per token row
+// per K block; the pitch is an odd number of 16-byte units so that the threads' vector reads of
+// their own slots do not collide in the banks
+__host__ __device__ constexpr int a_slot_pitch(int bits) { return bits == 3 ? 48 : 16 * bits + 16; }
 __host__ __device__ constexpr int n_a_stages(int bits) { return bits == 8 ? 2 : 4; }
 
 struct SmemLayout {
@@ -58,7 +59,7 @@ __host__ __device__ constexpr SmemLayout smem_layout(int ncta, int bits)
     SmemLayout s{};
     s.u_stage = A8_BYTES + w_rows(ncta) * KBLK;
     s.p_stage = w_rows(ncta) * KBLK / 2;
-    s.a_stage = 512 * a_slot_bytes(bits);
+    s.a_stage = TILE_M * a_slot_pitch(bits);
     s.off_p = n_u_stages(ncta) * s.u_stage;
     s.off_a = s.off_p + n_p_stages(ncta) * s.p_stage;
     s.off_flags = s.off_a + n_a_stages(bits) * s.a_stage;
@@ -163,13 +164,8 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
         "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
         ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
-// Asynchronous global -> shared copies of 4 or 16 bytes issued by ordinary threads; `valid` false
-// writes zeros and reads nothing.
-__device__ __forceinline__ void cp_async4(uint32_t dst, const void* src, bool valid)
-{
-    const uint32_t n = valid ? 4u : 0u;
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(n) : "memory");
-}
+// Asynchronous 16-byte global -> shared copy issued by an ordinary thread; `valid` false writes
+// zeros and reads nothing.
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool valid)
 {
     const uint32_t n = valid ? 16u : 0u;
@@ -402,40 +398,33 @@ cluster_gemm_kernel(const Params p)
         const int ut = tid - UNPACK_WARP0 * 32;      // 0..127
         uint32_t n_done = 0;
         const int total_kb = ((p.n_tiles - pair_id + n_pairs - 1) / n_pairs) * p.n_kb;
-        // Item i of this thread is row (ut >> 2) + 32 i, unit ut & 3, so its two chunk positions in
+        // Weight item i of this thread is row (ut >> 2) + 32 i, unit ut & 3, so its two chunk positions in
         // the swizzled row (16-byte chunk j of row r lives at position j ^ (r & 7)) are the same for every i.
         const int row0 = ut >> 2, unit = ut & 3, sw = row0 & 7;
         const uint32_t off0 = row0 * 128 + (((2 * unit) ^ sw) << 4), off1 = row0 * 128 + (((2 * unit + 1) ^ sw) << 4);
         constexpr int W_ITEMS = W_ROWS * 4 / 128;    // weight items per thread
-        // Activation codes: my four items of a K block are BITS words each, at rows m0 + row0 + 32 i,
-        // byte offset kb * 16 BITS + unit * 4 BITS of the row. They are fetched N_A - 1 K blocks ahead
-        // into slots that only this thread reads, so no other thread has to be waited for.
-        constexpr int N_A = n_a_stages(BITS), SLOT = a_slot_bytes(BITS);
-        const uint32_t a_ring = smem_base + SL.off_a + ut * SLOT;
-        auto fetch_a = [&](int t, int kb, int stage) {
-            const int m0 = (t % p.tiles_m) * (TILE_M * NCTA) + (int)cta_rank * TILE_M;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int row = m0 + row0 + 32 * i;
-                const bool valid = row < p.M;
-                const uint8_t* src = p.a_codes + (int64_t)(valid ? row : 0) * p.a_row_bytes + kb * (16 * BITS) + unit * (4 * BITS);
-                const uint32_t dst = a_ring + stage * SL.a_stage + i * 128 * SLOT;
-                if constexpr (BITS == 3) {
-#pragma unroll
-                    for (int j = 0; j < 3; ++j) cp_async4(dst + 4 * j, src + 4 * j, valid);
-                } else if constexpr (BITS == 4) {
-                    cp_async16(dst, src, valid);
-                } else {
-                    cp_async16(dst, src, valid);
-                    cp_async16(dst + 16, src + 16, valid);
-                }
-            }
+        // Activation codes: this thread owns token row `ut` of the tile. A K block of its row is
+        // 16 BITS contiguous bytes, fetched N_A - 1 K blocks ahead with 16-byte cp.async into a slot
+        // that only this thread reads, so no other thread has to be waited for.
+        constexpr int N_A = n_a_stages(BITS), PITCH = a_slot_pitch(BITS);
+        const uint32_t a_ring = smem_base + SL.off_a + ut * PITCH;
+        const uint32_t a_off = ut * 128, a_sw = ut & 7;          // my operand row and its swizzle
+        int t_f = pair_id, kb_f = 0, n_fetched = 0;             // next K block to fetch
+        const uint8_t* a_src = p.a_codes;                       // my row of the tile being fetched
+        bool a_ok = false;
+        auto fetch_tile_row = [&]() {
+            const int row = (t_f % p.tiles_m) * (TILE_M * NCTA) + (int)cta_rank * TILE_M + ut;
+            a_ok = row < p.M;
+            a_src = p.a_codes + (int64_t)(a_ok ? row : 0) * p.a_row_bytes;
         };
-        int t_f = pair_id, kb_f = 0, n_fetched = 0;      // next K block to fetch
+        fetch_tile_row();
         auto fetch_next = [&]() {
             if (n_fetched < total_kb) {
-                fetch_a(t_f, kb_f, n_fetched % N_A);
-                if (++kb_f == p.n_kb) { kb_f = 0; t_f += n_pairs; }
+                const uint32_t dst = a_ring + (n_fetched % N_A) * SL.a_stage;
+#pragma unroll
+                for (int j = 0; j < BITS; ++j) cp_async16(dst + 16 * j, a_src + 16 * j, a_ok);
+                a_src += 16 * BITS;
+                if (++kb_f == p.n_kb) { kb_f = 0; t_f += n_pairs; fetch_tile_row(); }
             }
             ++n_fetched;
             cp_async_commit();                           // one group per K block, empty past the end
@@ -446,19 +435,19 @@ cluster_gemm_kernel(const Params p)
             const int sp = n_done % N_P, su = n_done % N_U;
             fetch_next();
             cp_async_wait<N_A - 1>();                    // the group of K block `it` has landed
-            uint32_t pa_w[4][BITS];
+            uint32_t pa_w[4][BITS];                      // [unit][word]: unit u of the row is words BITS u ..
             {
                 const uint32_t slot = a_ring + (it % N_A) * SL.a_stage;
+                uint32_t raw[4 * BITS];
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const uint4 v = lds128(slot + i * 128 * SLOT);
-                    if constexpr (BITS == 3) { pa_w[i][0] = v.x; pa_w[i][1] = v.y; pa_w[i][2] = v.z; }
-                    else { pa_w[i][0] = v.x; pa_w[i][1] = v.y; pa_w[i][2] = v.z; pa_w[i][3] = v.w; }
-                    if constexpr (BITS == 8) {
-                        const uint4 u = lds128(slot + i * 128 * SLOT + 16);
-                        pa_w[i][4] = u.x; pa_w[i][5] = u.y; pa_w[i][6] = u.z; pa_w[i][7] = u.w;
-                    }
+                for (int j = 0; j < BITS; ++j) {
+                    const uint4 v = lds128(slot + 16 * j);
+                    raw[4 * j] = v.x; raw[4 * j + 1] = v.y; raw[4 * j + 2] = v.z; raw[4 * j + 3] = v.w;
                 }
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+#pragma unroll
+                    for (int j = 0; j < BITS; ++j) pa_w[u][j] = raw[BITS * u + j];
             }
             if (!mbar_wait(bar(B_PFULL + sp), (n_done / N_P) & 1, s_abort)) break;
             if (!mbar_wait(bar(B_UEMPTY + su), ((n_done / N_U) & 1) ^ 1, s_abort)) break;
@@ -473,11 +462,11 @@ cluster_gemm_kernel(const Params p)
                 pw_w[i][0] = v.x; pw_w[i][1] = v.y; pw_w[i][2] = v.z; pw_w[i][3] = v.w;
             }
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
+            for (int u = 0; u < 4; ++u) {
                 uint32_t o[8];
-                unpack_act32<BITS>(pa_w[i], o);
-                sts128(a_tile + off0 + i * 4096, o[0], o[1], o[2], o[3]);
-                sts128(a_tile + off1 + i * 4096, o[4], o[5], o[6], o[7]);
+                unpack_act32<BITS>(pa_w[u], o);
+                sts128(a_tile + a_off + (((2 * u) ^ a_sw) << 4), o[0], o[1], o[2], o[3]);
+                sts128(a_tile + a_off + (((2 * u + 1) ^ a_sw) << 4), o[4], o[5], o[6], o[7]);
             }
 #pragma unroll
             for (int i = 0; i < W_ITEMS; ++i) {
