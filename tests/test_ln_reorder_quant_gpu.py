@@ -117,7 +117,7 @@ def test_wide_rows_take_the_multi_unit_path_and_zero_tokens_launch_nothing():
     from paper_2304_01089_b200 import binding
     import torch
     rng = np.random.default_rng(11)
-    C, g, bits, M = 16384, 40, 4, 9
+    C, g, bits, M = 13312, 256, 4, 9
     perm, size, scale, zero = random_layout_params(rng, C, g, bits)
     L = binding.Layout(perm, size, scale, zero, bits)
     assert L.K_pad // 32 > 512
