@@ -81,6 +81,7 @@ struct Params {
     const uint8_t* step_flags;
     const float* seg_scale;
     const float* cl_sz;
+    const float* corr;           // optional [N]: sum_c s_c z_c Wsum_c[n] computed beforehand, else NULL
     const float* s_w;
     const int32_t* wsum;
     int64_t ld_w;
@@ -495,7 +496,8 @@ cluster_gemm_kernel(const Params p)
                 const int n = n0 + et;
                 float corr = 0.f, sw = 0.f, bs = 0.f;
                 if (n < p.N) {
-                    for (int c = 0; c < p.g; ++c) corr = __fmaf_rn(s_cl_sz[c], (float)__ldg(p.wsum + (int64_t)c * p.ld_w + n), corr);
+                    if (p.corr) corr = __ldg(p.corr + n);
+                    else for (int c = 0; c < p.g; ++c) corr = __fmaf_rn(s_cl_sz[c], (float)__ldg(p.wsum + (int64_t)c * p.ld_w + n), corr);
                     sw = __ldg(p.s_w + n);
                     bs = p.bias ? __ldg(p.bias + n) : 0.f;
                 }
@@ -644,9 +646,10 @@ static int launch(const Params& p, int n_sm, cudaStream_t st)
 
 using namespace rptq;
 
-extern "C" int rptq_cluster_gemm(const rptq_layout_t* Lin, const void* a_codes, int M, const void* w_codes,
-                                 const float* s_w, const int32_t* wsum, int64_t ld_w, const void* bias, int N,
-                                 int act, const rptq_layout_t* Lout, void* y, int y_dtype, int64_t ldy, void* stream)
+// Argument checks shared by the entry points. Returns RPTQ_OK when a launch should follow.
+static int check_gemm_args(const rptq_layout_t* Lin, const void* a_codes, int M, const void* w_codes,
+                           const float* s_w, const int32_t* wsum, int64_t ld_w, const void* bias, int N,
+                           int act, const rptq_layout_t* Lout, void* y, int y_dtype, int64_t ldy, int* dev_out)
 {
     if (!Lin || !a_codes || !w_codes || !s_w || !wsum || !y) return RPTQ_ERR_INVALID_ARG;
     if (M < 0 || N <= 0 || ld_w < N) return RPTQ_ERR_INVALID_ARG;
@@ -666,8 +669,16 @@ extern "C" int rptq_cluster_gemm(const rptq_layout_t* Lin, const void* a_codes, 
     int dev = -1;
     if (Lin->device < 0 || cudaGetDevice(&dev) != cudaSuccess) return RPTQ_ERR_CUDA;
     if (dev != Lin->device || (Lout && Lout->device != dev)) return RPTQ_ERR_INVALID_ARG;
-    if (M == 0) return RPTQ_OK;
+    *dev_out = dev;
+    return RPTQ_OK;
+}
 
+// Fills the launch parameters and launches the variant that fits M. `status` and `corr` may be NULL.
+static int launch_gemm(const rptq_layout_t* Lin, const void* a_codes, int M, const void* w_codes,
+                       const float* s_w, const int32_t* wsum, int64_t ld_w, const void* bias, int N,
+                       int act, const rptq_layout_t* Lout, void* y, int y_dtype, int64_t ldy, void* stream,
+                       int dev, int* status, const float* corr)
+{
     gemm::Params p{};
     p.M = M; p.N = N; p.n_kb = Lin->K_pad / gemm::KBLK; p.n_seg = Lin->n_seg; p.g = Lin->g;
     // CTA pairs share a 256-row tile; one token tile or less gains nothing from pairing
@@ -682,8 +693,8 @@ extern "C" int rptq_cluster_gemm(const rptq_layout_t* Lin, const void* a_codes, 
     p.out_unit = Lout ? Lout->d_unit : nullptr;
     p.out_bits = Lout ? Lout->bits : 0;
     p.out_row_bytes = Lout ? Lout->row_bytes : 0;
-    p.status = device_status_word();
-    if (!p.status) return RPTQ_ERR_ALLOC;
+    p.status = status;
+    p.corr = corr;
 
     int n_sm = 0;
     if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return RPTQ_ERR_CUDA;
@@ -697,3 +708,17 @@ extern "C" int rptq_cluster_gemm(const rptq_layout_t* Lin, const void* a_codes, 
     if (Lin->bits == 4) return gemm::launch<4, 1>(p, n_sm, st);
     return gemm::launch<8, 1>(p, n_sm, st);
 }
+
+extern "C" int rptq_cluster_gemm(const rptq_layout_t* Lin, const void* a_codes, int M, const void* w_codes,
+                                 const float* s_w, const int32_t* wsum, int64_t ld_w, const void* bias, int N,
+                                 int act, const rptq_layout_t* Lout, void* y, int y_dtype, int64_t ldy, void* stream)
+{
+    int dev = -1;
+    const int rc = check_gemm_args(Lin, a_codes, M, w_codes, s_w, wsum, ld_w, bias, N, act, Lout, y, y_dtype, ldy, &dev);
+    if (rc != RPTQ_OK) return rc;
+    if (M == 0) return RPTQ_OK;
+    int* status = device_status_word();
+    if (!status) return RPTQ_ERR_ALLOC;
+    return launch_gemm(Lin, a_codes, M, w_codes, s_w, wsum, ld_w, bias, N, act, Lout, y, y_dtype, ldy, stream, dev, status, nullptr);
+}
+
