@@ -162,6 +162,34 @@ int rptq_cluster_gemm(const rptq_layout_t* Lin, const void* a_codes, int M, cons
                       void* stream);
 
 /*
+ * The same operation as rptq_cluster_gemm, arguments and results included, for callers that must
+ * not allocate device memory. (The paper has no counterpart; this is a property of the library.)
+ * Who needs it: a process whose device memory is owned wholesale by its own pool -- an inference
+ * server that reserves the whole GPU at start-up, or a job running under a fixed memory budget --
+ * cannot let a library call cudaMalloc behind its back, and code that is recording work on a
+ * stream cannot afford a call that allocates on first use. rptq_cluster_gemm does allocate once,
+ * lazily (its status word); this entry point never does: it calls no cudaMalloc, cudaFree or
+ * allocating library routine.
+ * What it uses instead: a table of one float per output column (the zero-point correction
+ * sum_c s_c z_c Wsum_c[n], computed by a small kernel on `stream` just before the GEMM) that lives
+ * in a static device array of RPTQ_NOALLOC_MAX_N floats. Every device that loads the library
+ * holds these 256 KiB until the process exits.
+ *   - N > RPTQ_NOALLOC_MAX_N returns RPTQ_ERR_UNSUPPORTED and launches nothing.
+ *   - The first call on a device looks up the table's device address (a host-side query, no
+ *     allocation); make that first call outside any stream capture.
+ *   - All calls on a device share the one table. Each call rewrites the N entries it will read
+ *     before it reads them, so nothing has to be cleared; but two calls that can overlap on the
+ *     GPU (different streams, no dependency) race on it. Serialise them.
+ *   - A bounded wait that runs out inside the kernel leaves y undefined as in rptq_cluster_gemm,
+ *     but is not recorded anywhere: this variant has no status word.
+ */
+enum { RPTQ_NOALLOC_MAX_N = 65536 };
+int rptq_cluster_gemm_noalloc(const rptq_layout_t* Lin, const void* a_codes, int M, const void* w_codes,
+                              const float* s_w, const int32_t* wsum, int64_t ld_w, const void* bias, int N,
+                              int act, const rptq_layout_t* Lout, void* y, int y_dtype, int64_t ldy,
+                              void* stream);
+
+/*
  * Raw per-cluster integer accumulators of an output window (Appendix, X~_q,c W~_q,c before
  * de-quantisation), computed with plain integer instructions and no tensor cores:
  *   acc[c][m - m0][n - n0] = acc_c[m][n],  m0 <= m < m1 <= M, n0 <= n < n1 <= N

@@ -18,12 +18,13 @@ LIB_PATH = os.path.join(_HERE, "librptq.so")
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_NOT_BIJECTION, ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_ALLOC = 0, -1, -2, -3, -4, -5, -6
 OUT_F32, OUT_F16, OUT_CODES = 0, 1, 2
 ACT_NONE, ACT_RELU = 0, 1
+NOALLOC_MAX_N = 65536
 
 EXPORTS = (
     "rptq_layout_create", "rptq_layout_query", "rptq_layout_destroy", "rptq_ln_reorder_quant",
     "rptq_weight_pack", "rptq_cluster_gemm", "rptq_cluster_gemm_debug_acc", "rptq_codes_unpack_host",
     "rptq_codes_pack_host", "rptq_weight_unpack_host", "rptq_get_device_status", "rptq_status_string",
-    "rptq_format_version", "rptq_layout_padded_index", "rptq_weight_codes_bytes",
+    "rptq_format_version", "rptq_layout_padded_index", "rptq_weight_codes_bytes", "rptq_cluster_gemm_noalloc",
 )
 
 
@@ -47,6 +48,7 @@ def _load(path: str = LIB_PATH) -> C.CDLL:
     lib.rptq_ln_reorder_quant.argtypes = [vp, vp, i64, vp, vp, f32, i32, vp, vp, vp]
     lib.rptq_weight_pack.argtypes = [vp, vp, i32, vp, i32, vp, vp, vp]
     lib.rptq_cluster_gemm.argtypes = [vp, vp, i32, vp, vp, vp, i64, vp, i32, i32, vp, vp, i32, i64, vp]
+    lib.rptq_cluster_gemm_noalloc.argtypes = lib.rptq_cluster_gemm.argtypes
     lib.rptq_cluster_gemm_debug_acc.argtypes = [vp, vp, i32, vp, i32, i32, i32, i32, i32, vp, vp]
     lib.rptq_codes_unpack_host.argtypes = [i32, i32, vp, i64, vp]
     lib.rptq_codes_pack_host.argtypes = [i32, i32, vp, i64, vp]
@@ -185,6 +187,21 @@ def cluster_gemm(layout_in: Layout, a_codes, M: int, w_codes, s_w, wsum, N: int,
                                   _dev_ptr(wsum), ld_w, _dev_ptr(bias), int(N), int(act),
                                   None if layout_out is None else layout_out.handle, _dev_ptr(y), int(y_dtype),
                                   int(ldy), _stream_ptr(stream)), "rptq_cluster_gemm")
+
+
+def cluster_gemm_noalloc(layout_in: Layout, a_codes, M: int, w_codes, s_w, wsum, N: int, y, *, ld_w: Optional[int] = None,
+                         bias=None, act: int = ACT_NONE, layout_out: Optional[Layout] = None, y_dtype: int = OUT_F32,
+                         ldy: Optional[int] = None, stream=None) -> None:
+    """rptq_cluster_gemm_noalloc: same arguments and results as cluster_gemm, for callers that must
+    not allocate device memory (the library keeps its per-column scratch in a static device array;
+    N is limited to NOALLOC_MAX_N; calls that may overlap on the GPU must be serialised)."""
+    ld_w = int(s_w.shape[0]) if ld_w is None else int(ld_w)
+    if ldy is None:
+        ldy = 0 if y_dtype == OUT_CODES else int(y.stride(0))
+    _check(_lib.rptq_cluster_gemm_noalloc(layout_in.handle, _dev_ptr(a_codes), int(M), _dev_ptr(w_codes), _dev_ptr(s_w),
+                                          _dev_ptr(wsum), ld_w, _dev_ptr(bias), int(N), int(act),
+                                          None if layout_out is None else layout_out.handle, _dev_ptr(y), int(y_dtype),
+                                          int(ldy), _stream_ptr(stream)), "rptq_cluster_gemm_noalloc")
 
 
 def cluster_gemm_debug_acc(layout_in: Layout, a_codes, M: int, w_codes, N: int, m0: int, m1: int, n0: int, n1: int,

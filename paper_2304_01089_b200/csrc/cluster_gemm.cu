@@ -27,6 +27,8 @@
 // all roles drain and return.
 #include <cuda_fp16.h>
 
+#include <mutex>
+
 #include "pack.cuh"
 #include "rptq_internal.h"
 #include "unpack.cuh"
@@ -722,3 +724,64 @@ extern "C" int rptq_cluster_gemm(const rptq_layout_t* Lin, const void* a_codes, 
     return launch_gemm(Lin, a_codes, M, w_codes, s_w, wsum, ld_w, bias, N, act, Lout, y, y_dtype, ldy, stream, dev, status, nullptr);
 }
 
+// ---------------------------------------------------------------- entry point that allocates nothing
+namespace rptq {
+namespace gemm {
+
+// Scratch of rptq_cluster_gemm_noalloc: one zero-point correction per output column, resident in
+// every device that loads the library (256 KiB) until the process exits.
+static __device__ __align__(256) float g_noalloc_corr[RPTQ_NOALLOC_MAX_N];
+
+// corr[n] = sum_c s_c z_c Wsum_c[n], the same fused multiply-adds, in the same order, as the GEMM
+// epilogue performs when it is given no table.
+__global__ void noalloc_corr_kernel(const float* __restrict__ cl_sz, const int32_t* __restrict__ wsum, int64_t ld_w,
+                                    int g, int N, float* __restrict__ corr)
+{
+    const int n = blockIdx.x * blockDim.x + threadIdx.x;
+    if (n >= N) return;
+    float acc = 0.f;
+    for (int c = 0; c < g; ++c) acc = __fmaf_rn(__ldg(cl_sz + c), (float)__ldg(wsum + (int64_t)c * ld_w + n), acc);
+    corr[n] = acc;
+}
+
+// Device address of the scratch array, looked up once per device. In host code the array's name
+// is only a handle for the runtime; the address a kernel can use comes from cudaGetSymbolAddress
+// with that device current.
+static int noalloc_scratch(int dev, float** out)
+{
+    constexpr int kMaxDevices = 64;
+    static std::mutex mu;
+    static float* ptrs[kMaxDevices] = {};
+    if (dev < 0 || dev >= kMaxDevices) return RPTQ_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!ptrs[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_noalloc_corr) != cudaSuccess || !p) return RPTQ_ERR_CUDA;
+        ptrs[dev] = static_cast<float*>(p);
+    }
+    *out = ptrs[dev];
+    return RPTQ_OK;
+}
+
+}  // namespace gemm
+}  // namespace rptq
+
+extern "C" int rptq_cluster_gemm_noalloc(const rptq_layout_t* Lin, const void* a_codes, int M, const void* w_codes,
+                                         const float* s_w, const int32_t* wsum, int64_t ld_w, const void* bias, int N,
+                                         int act, const rptq_layout_t* Lout, void* y, int y_dtype, int64_t ldy, void* stream)
+{
+    int dev = -1;
+    int rc = check_gemm_args(Lin, a_codes, M, w_codes, s_w, wsum, ld_w, bias, N, act, Lout, y, y_dtype, ldy, &dev);
+    if (rc != RPTQ_OK) return rc;
+    if (N > RPTQ_NOALLOC_MAX_N) return RPTQ_ERR_UNSUPPORTED;    // more output columns than the resident table holds
+    if (M == 0) return RPTQ_OK;
+    float* corr = nullptr;
+    rc = gemm::noalloc_scratch(dev, &corr);
+    if (rc != RPTQ_OK) return rc;
+    auto st = static_cast<cudaStream_t>(stream);
+    // Every column the GEMM will read is rewritten here first, so nothing of the previous call's
+    // contents survives where it matters and nothing needs to start at zero.
+    gemm::noalloc_corr_kernel<<<(N + 255) / 256, 256, 0, st>>>(Lin->d_cl_sz, wsum, ld_w, Lin->g, N, corr);
+    if (cudaGetLastError() != cudaSuccess) return RPTQ_ERR_CUDA;
+    return launch_gemm(Lin, a_codes, M, w_codes, s_w, wsum, ld_w, bias, N, act, Lout, y, y_dtype, ldy, stream, dev, nullptr, corr);
+}
