@@ -28,6 +28,11 @@ sys.path.insert(0, ROOT)
 
 WORKLOAD = "opt-66b"
 EPS = 1e-5
+# dram__bytes_read + dram__bytes_write of one FC1 GEMM launch at 4096 tokens, from the ncu capture
+# summarised in profiles/cluster_gemm_opt66b_fc1_tokens512.txt: measured at 512 tokens (191.6 MB read,
+# of which 186.4 MB are the packed weights, read once whatever the token count) with the
+# token-proportional parts (codes in, fp16 output) scaled by 8.
+FC1_DRAM_BYTES_PER_LAUNCH = 186.4e6 + 8 * 5.2e6 + 8 * 37.7e6
 
 
 def _peaks():
@@ -235,7 +240,7 @@ def run_ours(args):
                 "cluster_gemm_fc1": {"ms": fc1_ms, "TOPS": achieved},
             },
             "roofline": {"bound": "tensor", "achieved": achieved, "peak": int8_peak, "unit": "TOP/s",
-                         "frac": achieved / int8_peak, "traffic": None,
+                         "frac": achieved / int8_peak, "traffic": FC1_DRAM_BYTES_PER_LAUNCH if M == w.tokens else None,
                          "kernel": "cluster_gemm_kernel<3> 4096x9216x36864",
                          "peak_note": f"2 x bf16 sustained ({peaks['source']})"},
             "e2e": None if args.no_e2e else {"value": world * ops_per_step * e2e_steps / (e2e_ms * 1e-3) / 1e12, "unit": "TOPS",
