@@ -17,7 +17,8 @@
 //               activation codes of a K block are 48/64/128 bytes per token row, too narrow for the
 //               copy engine to move at speed (measured: ~10 clk per row), so each unpack thread
 //               fetches the words of its own items with cp.async into a private ring of
-//               shared-memory slots, several K blocks ahead
+//               shared-memory slots, several K blocks ahead. 8-bit codes need no unpacking: with
+//               CTA pairs they are copied straight into the operand stage (template flag A8)
 //   warp 1      MMA issuer: four tcgen05.mma (K = 32 each) per K block; each cluster segment
 //               accumulates into one of two 256-column TMEM buffers and is committed when it ends
 //   warps 8-15  epilogue: drain a finished cluster's accumulator (tcgen05.ld), add s_c * acc into
@@ -46,7 +47,7 @@ constexpr long long WAIT_BUDGET_CYCLES = 4000000000ll;   // about two seconds at
 
 __host__ __device__ constexpr int w_rows(int ncta) { return TILE_N / ncta; }           // weight rows staged per CTA
 __host__ __device__ constexpr int n_p_stages(int ncta) { return ncta == 2 ? 4 : 3; }    // packed weight stages
-__host__ __device__ constexpr int n_u_stages(int ncta) { return ncta == 2 ? 4 : 2; }    // operand stages
+__host__ __device__ constexpr int n_u_stages(int ncta, bool a8) { return ncta == 2 ? (a8 ? 5 : 4) : 2; }   // operand stages
 // ring of packed activation K blocks fetched ahead by the unpack threads: one slot per token row
 // per K block; the pitch is an odd number of 16-byte units so that the threads' vector reads of
 // their own slots do not collide in the banks
@@ -56,13 +57,13 @@ __host__ __device__ constexpr int n_a_stages(int bits) { return bits == 8 ? 2 : 
 struct SmemLayout {
     int u_stage, p_stage, a_stage, off_p, off_a, off_flags, off_seg_scale, off_cl_sz, off_tab, off_bar, total;
 };
-__host__ __device__ constexpr SmemLayout smem_layout(int ncta, int bits)
+__host__ __device__ constexpr SmemLayout smem_layout(int ncta, int bits, bool a8)
 {
     SmemLayout s{};
     s.u_stage = A8_BYTES + w_rows(ncta) * KBLK;
     s.p_stage = w_rows(ncta) * KBLK / 2;
-    s.a_stage = TILE_M * a_slot_pitch(bits);
-    s.off_p = n_u_stages(ncta) * s.u_stage;
+    s.a_stage = a8 ? 0 : TILE_M * a_slot_pitch(bits);      // 8-bit activations go straight to the operand stage
+    s.off_p = n_u_stages(ncta, a8) * s.u_stage;
     s.off_a = s.off_p + n_p_stages(ncta) * s.p_stage;
     s.off_flags = s.off_a + n_a_stages(bits) * s.a_stage;
     s.off_seg_scale = s.off_flags + 2048;
@@ -249,14 +250,14 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr)
     return v;
 }
 
-template <int BITS, int NCTA>
+template <int BITS, int NCTA, bool A8>
 __global__ void __launch_bounds__(THREADS, 1)
 cluster_gemm_kernel(const Params p)
 {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
-    constexpr SmemLayout SL = smem_layout(NCTA, BITS);
+    constexpr SmemLayout SL = smem_layout(NCTA, BITS, A8);
     constexpr int W_ROWS = w_rows(NCTA);                 // weight rows this CTA stages and unpacks
-    constexpr int N_P = n_p_stages(NCTA), N_U = n_u_stages(NCTA);
+    constexpr int N_P = n_p_stages(NCTA), N_U = n_u_stages(NCTA, A8);
     constexpr uint32_t kInstrDesc = instr_desc(NCTA);
     // dynamic shared memory is only guaranteed 16-byte alignment: round up to the swizzle span
     // (the offset is the same in both CTAs of a pair, as cta_group::2 descriptors require)
@@ -356,14 +357,15 @@ cluster_gemm_kernel(const Params p)
             const uint64_t a_desc0 = smem_desc_sw128(smem_base), w_desc0 = smem_desc_sw128(smem_base + A8_BYTES);
             const uint32_t* flags4 = reinterpret_cast<const uint32_t*>(s_flags);
             uint32_t d_tmem = tmem_base;
+            uint32_t f4 = flags4[0];
             for (int t = pair_id; t < p.n_tiles && ok; t += n_pairs) {
                 for (int kb = 0; kb < p.n_kb && ok; ++kb, ++n_kb_done) {
                     const int s = n_kb_done % N_U;
+                    const uint32_t f4_next = flags4[kb + 1 < p.n_kb ? kb + 1 : 0];    // read while waiting
                     if (!mbar_wait(bar(B_UFULL + s), (n_kb_done / N_U) & 1, s_abort)) { ok = false; break; }
                     tc_fence_after();
                     // the start-address field counts 16-byte units: one stage further, 32 bytes per step
                     const uint64_t ad = a_desc0 + (uint64_t)(s * (SL.u_stage >> 4)), wd = w_desc0 + (uint64_t)(s * (SL.u_stage >> 4));
-                    const uint32_t f4 = flags4[kb];
                     if (f4 == 0) {
                         tc_mma_i8<NCTA>(d_tmem, ad, wd, kInstrDesc, 1u);
                         tc_mma_i8<NCTA>(d_tmem, ad + 2, wd + 2, kInstrDesc, 1u);
@@ -373,6 +375,7 @@ cluster_gemm_kernel(const Params p)
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
                             const uint32_t f = (f4 >> (8 * j)) & 0xFFu;
+                            if (f == 0) { tc_mma_i8<NCTA>(d_tmem, ad + 2 * j, wd + 2 * j, kInstrDesc, 1u); continue; }   // inside a cluster
                             if (f & STEP_SKIP) continue;
                             if (f & STEP_FIRST) {
                                 if (!mbar_wait(bar(B_ACCEMPTY + (n_seg_done & 1)), ((n_seg_done >> 1) & 1) ^ 1, s_abort)) { ok = false; break; }
@@ -387,6 +390,7 @@ cluster_gemm_kernel(const Params p)
                         }
                     }
                     tc_commit<NCTA>(bar(B_UEMPTY + s));      // the stage may be overwritten once these MMAs have read it
+                    f4 = f4_next;
                 }
             }
             if (!ok) {
@@ -406,14 +410,82 @@ cluster_gemm_kernel(const Params p)
         const int row0 = ut >> 2, unit = ut & 3, sw = row0 & 7;
         const uint32_t off0 = row0 * 128 + (((2 * unit) ^ sw) << 4), off1 = row0 * 128 + (((2 * unit + 1) ^ sw) << 4);
         constexpr int W_ITEMS = W_ROWS * 4 / 128;    // weight items per thread
+        const uint32_t a_off = ut * 128, a_sw = ut & 7;          // my operand row and its swizzle
+        int t_f = pair_id, kb_f = 0, n_fetched = 0;             // next K block to fetch
+        const uint8_t* a_src = p.a_codes;
+        if constexpr (A8) {
+            // The codes are bytes already: a K block of a token row is 128 contiguous bytes. Eight
+            // lanes copy the eight 16-byte chunks of one row (one cache line per row, so a warp-wide
+            // cp.async touches 4 lines, not 32) straight into that row's swizzled place in the
+            // operand stage; a warp covers its 32 rows in eight such instructions, PF K blocks
+            // ahead of the weights. The stage is waited for (its previous MMAs have read it) first.
+            constexpr int PF = N_U - 2;
+            bool ok = true;
+            const int wrow = (warp - UNPACK_WARP0) * 32 + (lane >> 3), ch = lane & 7;   // rows wrow + 4 i, chunk ch
+            const uint32_t d_even = (uint32_t)wrow * 128 + ((ch ^ (lane >> 3)) << 4);
+            const uint32_t d_odd = (uint32_t)wrow * 128 + ((ch ^ ((lane >> 3) + 4)) << 4);
+            const int64_t step4 = 4 * p.a_row_bytes;
+            int n_rows_ok = 0;                               // how many of my 8 rows exist
+            auto a8_tile = [&]() {
+                const int row = (t_f % p.tiles_m) * (TILE_M * NCTA) + (int)cta_rank * TILE_M + wrow;
+                const int left = p.M - row;
+                n_rows_ok = left <= 0 ? 0 : (left + 3) >> 2;
+                a_src = p.a_codes + (int64_t)(left > 0 ? row : 0) * p.a_row_bytes + 16 * ch;
+            };
+            a8_tile();
+            auto fetch_next = [&]() {
+                if (n_fetched < total_kb && ok) {
+                    const int s2 = n_fetched % N_U;
+                    if (!mbar_wait(bar(B_UEMPTY + s2), ((n_fetched / N_U) & 1) ^ 1, s_abort)) { ok = false; }
+                    else {
+                        tc_fence_after();
+                        const uint32_t dst = smem_base + s2 * SL.u_stage;
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const bool v = i < n_rows_ok;
+                            cp_async16(dst + ((i & 1) ? d_odd : d_even) + i * 512, v ? a_src + i * step4 : p.a_codes, v);
+                        }
+                        a_src += KBLK;
+                        if (++kb_f == p.n_kb) { kb_f = 0; t_f += n_pairs; a8_tile(); }
+                    }
+                }
+                ++n_fetched;
+                cp_async_commit();                           // one group per K block, empty past the end
+            };
+#pragma unroll 1
+            for (int i = 0; i < PF; ++i) fetch_next();
+            for (int it = 0; it < total_kb && ok; ++it, ++n_done) {
+                const int sp = n_done % N_P, su = n_done % N_U;
+                fetch_next();
+                if (!ok) break;
+                if (!mbar_wait(bar(B_PFULL + sp), (n_done / N_P) & 1, s_abort)) break;
+                const uint32_t pw = smem_base + SL.off_p + sp * SL.p_stage;
+                const uint32_t w_tile = smem_base + su * SL.u_stage + A8_BYTES;
+                uint32_t pw_w[W_ITEMS][4];
+#pragma unroll
+                for (int i = 0; i < W_ITEMS; ++i) {
+                    const uint4 v = lds128(pw + (ut + i * 128) * 16);
+                    pw_w[i][0] = v.x; pw_w[i][1] = v.y; pw_w[i][2] = v.z; pw_w[i][3] = v.w;
+                }
+#pragma unroll
+                for (int i = 0; i < W_ITEMS; ++i) {
+                    uint32_t o[8];
+                    unpack_w32_x16(pw_w[i], o);
+                    sts128(w_tile + off0 + i * 4096, o[0], o[1], o[2], o[3]);
+                    sts128(w_tile + off1 + i * 4096, o[4], o[5], o[6], o[7]);
+                }
+                cp_async_wait<PF>();                         // my copies of K block `it` have landed
+                fence_proxy_async();          // make the generic-proxy writes visible to the tensor core
+                __syncwarp();                 // ... and every lane's copies and stores of this warp
+                if (lane == 0) { arrive_leader(bar(B_UFULL + su)); mbar_arrive(bar(B_PEMPTY + sp)); }
+            }
+            cp_async_wait<0>();
+        } else {
         // Activation codes: this thread owns token row `ut` of the tile. A K block of its row is
         // 16 BITS contiguous bytes, fetched N_A - 1 K blocks ahead with 16-byte cp.async into a slot
         // that only this thread reads, so no other thread has to be waited for.
         constexpr int N_A = n_a_stages(BITS), PITCH = a_slot_pitch(BITS);
         const uint32_t a_ring = smem_base + SL.off_a + ut * PITCH;
-        const uint32_t a_off = ut * 128, a_sw = ut & 7;          // my operand row and its swizzle
-        int t_f = pair_id, kb_f = 0, n_fetched = 0;             // next K block to fetch
-        const uint8_t* a_src = p.a_codes;                       // my row of the tile being fetched
         bool a_ok = false;
         auto fetch_tile_row = [&]() {
             const int row = (t_f % p.tiles_m) * (TILE_M * NCTA) + (int)cta_rank * TILE_M + ut;
@@ -481,6 +553,8 @@ cluster_gemm_kernel(const Params p)
             fence_proxy_async();          // make the generic-proxy stores visible to the tensor core
             __syncwarp();
             if (lane == 0) { arrive_leader(bar(B_UFULL + su)); mbar_arrive(bar(B_PEMPTY + sp)); }
+        }
+        cp_async_wait<0>();
         }
     } else {
         // ------------------------------------------------------------ epilogue warps
@@ -617,12 +691,12 @@ cluster_gemm_kernel(const Params p)
 }
 
 // ---------------------------------------------------------------- host side
-template <int BITS, int NCTA>
+template <int BITS, int NCTA, bool A8>
 static int launch(const Params& p, int n_sm, cudaStream_t st)
 {
-    constexpr SmemLayout SL = smem_layout(NCTA, BITS);
+    constexpr SmemLayout SL = smem_layout(NCTA, BITS, A8);
     const int smem = SL.total + 1024;     // slack for the in-kernel 1024-byte alignment
-    const void* fn = reinterpret_cast<const void*>(cluster_gemm_kernel<BITS, NCTA>);
+    const void* fn = reinterpret_cast<const void*>(cluster_gemm_kernel<BITS, NCTA, A8>);
     cudaFuncAttributes attr;
     if (cudaFuncGetAttributes(&attr, fn) != cudaSuccess) return RPTQ_ERR_CUDA;
     // the register re-partition inside the kernel (setmaxnreg) assumes this pool; refuse to launch otherwise
@@ -640,7 +714,7 @@ static int launch(const Params& p, int n_sm, cudaStream_t st)
     at[0].val.clusterDim.x = NCTA; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
     cfg.attrs = at;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, cluster_gemm_kernel<BITS, NCTA>, p) == cudaSuccess ? RPTQ_OK : RPTQ_ERR_CUDA;
+    return cudaLaunchKernelEx(&cfg, cluster_gemm_kernel<BITS, NCTA, A8>, p) == cudaSuccess ? RPTQ_OK : RPTQ_ERR_CUDA;
 }
 
 }  // namespace gemm
@@ -702,13 +776,13 @@ static int launch_gemm(const rptq_layout_t* Lin, const void* a_codes, int M, con
     if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return RPTQ_ERR_CUDA;
     auto st = static_cast<cudaStream_t>(stream);
     if (ncta == 2) {
-        if (Lin->bits == 3) return gemm::launch<3, 2>(p, n_sm, st);
-        if (Lin->bits == 4) return gemm::launch<4, 2>(p, n_sm, st);
-        return gemm::launch<8, 2>(p, n_sm, st);
+        if (Lin->bits == 3) return gemm::launch<3, 2, false>(p, n_sm, st);
+        if (Lin->bits == 4) return gemm::launch<4, 2, false>(p, n_sm, st);
+        return gemm::launch<8, 2, true>(p, n_sm, st);      // 8-bit codes need no unpacking
     }
-    if (Lin->bits == 3) return gemm::launch<3, 1>(p, n_sm, st);
-    if (Lin->bits == 4) return gemm::launch<4, 1>(p, n_sm, st);
-    return gemm::launch<8, 1>(p, n_sm, st);
+    if (Lin->bits == 3) return gemm::launch<3, 1, false>(p, n_sm, st);
+    if (Lin->bits == 4) return gemm::launch<4, 1, false>(p, n_sm, st);
+    return gemm::launch<8, 1, false>(p, n_sm, st);
 }
 
 extern "C" int rptq_cluster_gemm(const rptq_layout_t* Lin, const void* a_codes, int M, const void* w_codes,
