@@ -239,6 +239,15 @@ __host__ __device__ constexpr uint32_t instr_desc(int ncta)
     return (2u << 4) | (0u << 7) | (1u << 10) | ((uint32_t)(TILE_N >> 3) << 17) | ((uint32_t)((TILE_M * ncta) >> 4) << 24);
 }
 
+// packed fp32 pairs: one instruction, two independent IEEE results
+__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c)
+{
+    float2 d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(reinterpret_cast<uint64_t&>(d))
+        : "l"(reinterpret_cast<uint64_t&>(a)), "l"(reinterpret_cast<uint64_t&>(b)), "l"(reinterpret_cast<uint64_t&>(c)));
+    return d;
+}
+
 __device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
 {
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
@@ -564,7 +573,7 @@ cluster_gemm_kernel(const Params p)
         const int et = ew * 32 + lane;               // 0..255: the column whose tile constants I prepare
         uint32_t n_seg_done = 0, n_tile_done = 0;
         bool ok = true;
-        float R[128];
+        float2 R[64];                                // running sums of columns 2 i, 2 i + 1
         for (int t = pair_id; t < p.n_tiles && ok; t += n_pairs, ++n_tile_done) {
             const int m0 = (t % p.tiles_m) * (TILE_M * NCTA) + (int)cta_rank * TILE_M, n0 = (t / p.tiles_m) * TILE_N;
             float* tab = s_tab + (n_tile_done & 1) * 3 * TILE_N;
@@ -582,25 +591,30 @@ cluster_gemm_kernel(const Params p)
                 if (lane == 0) mbar_arrive(bar(B_TAB + (n_tile_done & 1)));
             }
 #pragma unroll
-            for (int i = 0; i < 128; ++i) R[i] = 0.f;
+            for (int i = 0; i < 64; ++i) R[i] = make_float2(0.f, 0.f);
             for (int sgi = 0; sgi < p.n_seg; ++sgi, ++n_seg_done) {
                 const uint32_t buf = n_seg_done & 1;
                 if (!mbar_wait(bar(B_ACCFULL + buf), (n_seg_done >> 1) & 1, s_abort)) { ok = false; break; }
                 tc_fence_after();
                 const float sc = s_seg_scale[sgi];
+                const float2 sc2 = make_float2(sc, sc);
                 const uint32_t taddr = tmem_base + ((uint32_t)(32 * q) << 16) + buf * TILE_N + h * 128;
                 uint32_t va[16], vb[16];
                 tc_ld16(taddr, va);
+                // R += s_c * acc, two columns per packed fused multiply-add
+                auto accumulate = [&](const uint32_t (&v)[16], int c0) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        R[c0 + i] = fma2(sc2, make_float2((float)(int)v[2 * i], (float)(int)v[2 * i + 1]), R[c0 + i]);
+                };
 #pragma unroll
                 for (int ch = 0; ch < 8; ch += 2) {
                     tc_wait_ld();
                     tc_ld16(taddr + (ch + 1) * 16, vb);
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) R[ch * 16 + i] = __fmaf_rn(sc, (float)(int)va[i], R[ch * 16 + i]);
+                    accumulate(va, ch * 8);
                     tc_wait_ld();
                     if (ch + 2 < 8) tc_ld16(taddr + (ch + 2) * 16, va);
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) R[(ch + 1) * 16 + i] = __fmaf_rn(sc, (float)(int)vb[i], R[(ch + 1) * 16 + i]);
+                    accumulate(vb, (ch + 1) * 8);
                 }
                 tc_fence_before();
                 __syncwarp();
@@ -614,29 +628,30 @@ cluster_gemm_kernel(const Params p)
             const float* t_corr = tab + h * 128;
             const float* t_sw = tab + TILE_N + h * 128;
             const float* t_bs = tab + 2 * TILE_N + h * 128;
+            auto Rf = [&](int i) -> float& { return (i & 1) ? R[i >> 1].y : R[i >> 1].x; };
 #pragma unroll
             for (int i = 0; i < 128; ++i) {
-                float v = __fmaf_rn(t_sw[i], R[i] - t_corr[i], t_bs[i]);
+                float v = __fmaf_rn(t_sw[i], Rf(i) - t_corr[i], t_bs[i]);
                 if (p.act == RPTQ_ACT_RELU) v = fmaxf(v, 0.f);
-                R[i] = v;
+                Rf(i) = v;
             }
             if (m < p.M) {
                 if (p.y_dtype == RPTQ_OUT_F32) {
                     float* dst = static_cast<float*>(p.y) + (int64_t)m * p.ldy + nb;
                     if (nb + 128 <= p.N) {
 #pragma unroll
-                        for (int i = 0; i < 128; i += 4) *reinterpret_cast<float4*>(dst + i) = make_float4(R[i], R[i + 1], R[i + 2], R[i + 3]);
+                        for (int i = 0; i < 128; i += 4) *reinterpret_cast<float4*>(dst + i) = make_float4(Rf(i), Rf(i + 1), Rf(i + 2), Rf(i + 3));
                     } else {
 #pragma unroll
-                        for (int i = 0; i < 128; ++i) if (nb + i < p.N) dst[i] = R[i];
+                        for (int i = 0; i < 128; ++i) if (nb + i < p.N) dst[i] = Rf(i);
                     }
                 } else if (p.y_dtype == RPTQ_OUT_F16) {
                     __half* dst = static_cast<__half*>(p.y) + (int64_t)m * p.ldy + nb;
                     if (nb + 128 <= p.N) {
 #pragma unroll
                         for (int i = 0; i < 128; i += 8) {
-                            __half2 h0 = __floats2half2_rn(R[i], R[i + 1]), h1 = __floats2half2_rn(R[i + 2], R[i + 3]);
-                            __half2 h2 = __floats2half2_rn(R[i + 4], R[i + 5]), h3 = __floats2half2_rn(R[i + 6], R[i + 7]);
+                            __half2 h0 = __floats2half2_rn(Rf(i), Rf(i + 1)), h1 = __floats2half2_rn(Rf(i + 2), Rf(i + 3));
+                            __half2 h2 = __floats2half2_rn(Rf(i + 4), Rf(i + 5)), h3 = __floats2half2_rn(Rf(i + 6), Rf(i + 7));
                             uint4 v;
                             v.x = *reinterpret_cast<uint32_t*>(&h0); v.y = *reinterpret_cast<uint32_t*>(&h1);
                             v.z = *reinterpret_cast<uint32_t*>(&h2); v.w = *reinterpret_cast<uint32_t*>(&h3);
@@ -644,7 +659,7 @@ cluster_gemm_kernel(const Params p)
                         }
                     } else {
 #pragma unroll
-                        for (int i = 0; i < 128; ++i) if (nb + i < p.N) dst[i] = __float2half_rn(R[i]);
+                        for (int i = 0; i < 128; ++i) if (nb + i < p.N) dst[i] = __float2half_rn(Rf(i));
                     }
                 } else {
                     // re-quantise for the next site: column n is padded position n of the output layout
@@ -659,7 +674,7 @@ cluster_gemm_kernel(const Params p)
                         const int zc = (int)t4.y, nvalid = (int)t4.w;
                         uint32_t qv[32];
 #pragma unroll
-                        for (int e = 0; e < 32; ++e) qv[e] = e < nvalid ? quant_code(R[32 * uu + e], inv_s, zc, qmax) : 0u;
+                        for (int e = 0; e < 32; ++e) qv[e] = e < nvalid ? quant_code(Rf(32 * uu + e), inv_s, zc, qmax) : 0u;
                         if (p.out_bits == 4) {
                             uint32_t w[4]; pack32<4>(qv, w);
                             *reinterpret_cast<uint4*>(row + unit * 16) = make_uint4(w[0], w[1], w[2], w[3]);
