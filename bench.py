@@ -100,7 +100,7 @@ def _prepare_site(sw, li, n_tokens, torch, binding):
     gamma, beta = workloads.ln_params(sw)
     cal = calibration.calibrate(workloads.calib_tokens(sw), gamma, beta, sw.clusters, sw.bits,
                                 workloads.kmeans_draws(sw, 0, sw.clusters), EPS)
-    L = binding.Layout(cal.perm, cal.size, cal.scale, cal.zero, sw.bits)
+    L = binding.Layout(cal.perm, cal.size, cal.scale, cal.zero, sw.bits, order=binding.ORDER_INTERLEAVED)
     n_out = sw.linears[li].n_out
     rb = L.K_pad // 2
     w_codes = np.zeros(binding.weight_codes_bytes(L.K_pad, n_out), np.uint8)

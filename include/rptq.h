@@ -25,11 +25,24 @@
  *   S = [S^1 .. S^g] the reorder index, n_c = |S^c|, (s_c, z_c) the quantisation parameters of
  *   cluster c.
  *
- * Padded segment layout (not in the paper; the tensor-core contraction step is 32 codes wide and
- * operands are staged in blocks of 128): in a row of codes cluster c occupies positions
- * seg_off[c] .. seg_off[c] + n_c - 1 with seg_off[c] = sum_{c' < c} roundup32(n_c'), and the row
- * length is K_pad = max(128, roundup128(seg_off[g])). Pad positions hold activation code 0 and
- * weight code 0.
+ * Padded layout (not in the paper; the tensor-core contraction step is 32 codes wide and operands
+ * are staged in blocks of 128): a row of codes is K_pad/32 units of 32 positions. Cluster c owns
+ * roundup32(n_c)/32 units; its channels fill them in the order of S, so only its last unit can
+ * hold pad positions (at the end). K_pad = max(128, roundup128(sum_c roundup32(n_c))); the units
+ * left over at the end of the row belong to no cluster. Pad positions hold activation code 0 and
+ * weight code 0. Two unit orders:
+ *   RPTQ_ORDER_CONTIGUOUS   the clusters' units follow one another in the order of S, so cluster
+ *                           c occupies positions seg_off[c] .. seg_off[c] + n_c - 1 with
+ *                           seg_off[c] = sum_{c' < c} roundup32(n_c');
+ *   RPTQ_ORDER_INTERLEAVED  clusters of one or two units are placed between the units of the
+ *                           larger clusters, one after every seven larger-cluster units (those left
+ *                           over follow at the end); a larger cluster's units keep their order
+ *                           but are no longer adjacent. The GEMM drains one accumulator per
+ *                           cluster, and a run of very small clusters leaves the tensor cores
+ *                           waiting for those drains; spread out, each drain runs under the
+ *                           surrounding cluster's products. Falls back to the contiguous order
+ *                           when there are fewer than two small clusters or no larger one.
+ * rptq_layout_query and rptq_layout_padded_index report where everything went.
  *
  * Packed storage, format version 2 (private to this library; read it back with the *_unpack_host
  * helpers). A row of K_pad codes takes K_pad*bits/8 bytes:
@@ -67,6 +80,7 @@ enum {
 enum { RPTQ_OUT_F32 = 0, RPTQ_OUT_F16 = 1, RPTQ_OUT_CODES = 2 };
 enum { RPTQ_ACT_NONE = 0, RPTQ_ACT_RELU = 1 };
 enum { RPTQ_FORMAT_VERSION = 2 };
+enum { RPTQ_ORDER_CONTIGUOUS = 0, RPTQ_ORDER_INTERLEAVED = 1 };
 
 typedef struct rptq_layout rptq_layout_t;
 
@@ -81,16 +95,19 @@ typedef struct rptq_layout rptq_layout_t;
  *   zero_host[g]     z_c for codes re-based to [0, 2^bits - 1] (Eq. 1 states the signed range
  *                    [-2^(k-1), 2^(k-1)-1]; adding 2^(k-1) to both code and zero point leaves
  *                    s (x_q - z) unchanged). |z_c| < 2^21.
+ *   order            RPTQ_ORDER_CONTIGUOUS or RPTQ_ORDER_INTERLEAVED (see "Padded layout" above).
+ *                    Codes, packed weights and layouts of different orders do not mix.
  * Limits: C a multiple of 8, 8 <= C <= 65528, 1 <= g <= 4096, K_pad <= 65408; otherwise
  * RPTQ_ERR_UNSUPPORTED. On success *out owns small device tables on the current device; free it
  * with rptq_layout_destroy. All four arrays are copied.
  */
 int rptq_layout_create(rptq_layout_t** out, int C, int g, int bits,
                        const int32_t* perm_host, const int32_t* cluster_size,
-                       const float* scale_host, const int32_t* zero_host);
+                       const float* scale_host, const int32_t* zero_host, int order);
 
-/* Sizes of the padded layout. Any output pointer may be NULL. seg_offset_out receives g+1 ints. */
-int rptq_layout_query(const rptq_layout_t* L, int* K_pad, int64_t* row_bytes, int32_t* seg_offset_out);
+/* Sizes of the padded layout. Any output pointer may be NULL. unit_cluster_out receives K_pad/32
+ * ints: the cluster that owns each unit of 32 positions, -1 for the units past the last cluster. */
+int rptq_layout_query(const rptq_layout_t* L, int* K_pad, int64_t* row_bytes, int32_t* unit_cluster_out);
 
 /* padded_index[K_pad]: the original channel held by each padded position, -1 for pad positions. */
 int rptq_layout_padded_index(const rptq_layout_t* L, int32_t* padded_index);

@@ -19,6 +19,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_NOT_BIJECTION, ERR_CUDA, ERR_DEVICE_TI
 OUT_F32, OUT_F16, OUT_CODES = 0, 1, 2
 ACT_NONE, ACT_RELU = 0, 1
 NOALLOC_MAX_N = 65536
+ORDER_CONTIGUOUS, ORDER_INTERLEAVED = 0, 1
 
 EXPORTS = (
     "rptq_layout_create", "rptq_layout_query", "rptq_layout_destroy", "rptq_ln_reorder_quant",
@@ -41,7 +42,7 @@ def _load(path: str = LIB_PATH) -> C.CDLL:
             "(nvcc, sm_100a). There is no CPU or PyTorch fallback.")
     lib = C.CDLL(path)
     vp, i32, i64, f32 = C.c_void_p, C.c_int, C.c_int64, C.c_float
-    lib.rptq_layout_create.argtypes = [C.POINTER(vp), i32, i32, i32, vp, vp, vp, vp]
+    lib.rptq_layout_create.argtypes = [C.POINTER(vp), i32, i32, i32, vp, vp, vp, vp, i32]
     lib.rptq_layout_query.argtypes = [vp, C.POINTER(i32), C.POINTER(i64), vp]
     lib.rptq_layout_destroy.argtypes = [vp]
     lib.rptq_layout_padded_index.argtypes = [vp, vp]
@@ -102,7 +103,7 @@ def _stream_ptr(stream) -> Optional[int]:
 class Layout:
     """rptq_layout_create / _query / _destroy: reorder index S, cluster sizes, (s_c, z_c)."""
 
-    def __init__(self, perm, cluster_size, scale, zero, bits: int):
+    def __init__(self, perm, cluster_size, scale, zero, bits: int, order: int = ORDER_CONTIGUOUS):
         self._perm = np.ascontiguousarray(perm, dtype=np.int32)
         self._size = np.ascontiguousarray(cluster_size, dtype=np.int32)
         self._scale = np.ascontiguousarray(scale, dtype=np.float32)
@@ -112,13 +113,15 @@ class Layout:
         self.C, self.g, self.bits = int(self._perm.shape[0]), int(self._size.shape[0]), int(bits)
         h = C.c_void_p()
         _check(_lib.rptq_layout_create(C.byref(h), self.C, self.g, self.bits, _np_ptr(self._perm),
-                                       _np_ptr(self._size), _np_ptr(self._scale), _np_ptr(self._zero)),
+                                       _np_ptr(self._size), _np_ptr(self._scale), _np_ptr(self._zero), int(order)),
                "rptq_layout_create")
         self._h = h
+        self.order = int(order)
         k_pad, rb = C.c_int(), C.c_int64()
-        self.seg_off = np.empty(self.g + 1, np.int32)
-        _check(_lib.rptq_layout_query(self._h, C.byref(k_pad), C.byref(rb), _np_ptr(self.seg_off)), "rptq_layout_query")
+        _check(_lib.rptq_layout_query(self._h, C.byref(k_pad), C.byref(rb), None), "rptq_layout_query")
         self.K_pad, self.row_bytes = int(k_pad.value), int(rb.value)
+        self.unit_cluster = np.empty(self.K_pad // 32, np.int32)      # owning cluster of each unit of 32 positions
+        _check(_lib.rptq_layout_query(self._h, None, None, _np_ptr(self.unit_cluster)), "rptq_layout_query")
 
     @property
     def handle(self) -> C.c_void_p:
@@ -130,6 +133,25 @@ class Layout:
         """int32 [K_pad]: original channel at each padded position, -1 at pads."""
         out = np.empty(self.K_pad, np.int32)
         _check(_lib.rptq_layout_padded_index(self.handle, _np_ptr(out)), "rptq_layout_padded_index")
+        return out
+
+    def contiguous_position(self) -> np.ndarray:
+        """int32 [K_pad]: for each position of this layout, the position that holds the same channel
+        (or pad) in the contiguous unit order, where cluster c starts at sum_{c' < c} roundup32(n_c').
+        A [*, K_pad] array `a` in contiguous order becomes `a[:, m]` in this layout's order."""
+        units = (self._size.astype(np.int64) + 31) // 32
+        first = np.concatenate([[0], np.cumsum(units)])
+        seen = np.zeros(self.g, np.int64)
+        tail = int(first[-1])
+        out = np.empty(self.K_pad, np.int32)
+        for u, c in enumerate(self.unit_cluster):
+            if c < 0:
+                cu = tail
+                tail += 1
+            else:
+                cu = int(first[c] + seen[c])
+                seen[c] += 1
+            out[32 * u:32 * u + 32] = np.arange(32 * cu, 32 * cu + 32)
         return out
 
     def destroy(self) -> None:

@@ -19,8 +19,12 @@
 //               fetches the words of its own items with cp.async into a private ring of
 //               shared-memory slots, several K blocks ahead. 8-bit codes need no unpacking: with
 //               CTA pairs they are copied straight into the operand stage (template flag A8)
-//   warp 1      MMA issuer: four tcgen05.mma (K = 32 each) per K block; each cluster segment
-//               accumulates into one of two 256-column TMEM buffers and is committed when it ends
+//   warp 1      MMA issuer: four tcgen05.mma (K = 32 each) per K block; each cluster accumulates
+//               into one of two 256-column TMEM buffers (the layout's step flags say which) and
+//               is committed at its last step. A cluster's steps need not be adjacent: in the
+//               interleaved unit order a small cluster's step sits between those of a large one,
+//               which keeps its buffer, so the small cluster's drain runs under the large
+//               cluster's remaining products
 //   warps 8-15  epilogue: drain a finished cluster's accumulator (tcgen05.ld), add s_c * acc into
 //               fp32 running sums held in registers while the next cluster's MMAs run; after the
 //               last cluster apply the zero-point correction, s_w, bias, activation, and store
@@ -55,7 +59,7 @@ __host__ __device__ constexpr int a_slot_pitch(int bits) { return bits == 3 ? 48
 __host__ __device__ constexpr int n_a_stages(int bits) { return bits == 8 ? 2 : 4; }
 
 struct SmemLayout {
-    int u_stage, p_stage, a_stage, off_p, off_a, off_flags, off_seg_scale, off_cl_sz, off_tab, off_bar, total;
+    int u_stage, p_stage, a_stage, off_p, off_a, off_flags, off_seg_scale, off_seg_buf, off_cl_sz, off_tab, off_bar, total;
 };
 __host__ __device__ constexpr SmemLayout smem_layout(int ncta, int bits, bool a8)
 {
@@ -67,7 +71,8 @@ __host__ __device__ constexpr SmemLayout smem_layout(int ncta, int bits, bool a8
     s.off_a = s.off_p + n_p_stages(ncta) * s.p_stage;
     s.off_flags = s.off_a + n_a_stages(bits) * s.a_stage;
     s.off_seg_scale = s.off_flags + 2048;
-    s.off_cl_sz = s.off_seg_scale + kMaxGemmSegments * 4;
+    s.off_seg_buf = s.off_seg_scale + kMaxGemmSegments * 4;
+    s.off_cl_sz = s.off_seg_buf + kMaxGemmSegments;
     s.off_tab = s.off_cl_sz + kMaxGemmSegments * 4;
     s.off_bar = s.off_tab + 2 * 3 * TILE_N * 4;
     s.total = s.off_bar + 256;
@@ -82,7 +87,8 @@ struct Params {
     const uint8_t* w_codes;      // tile-major: n_wtiles * n_kb tiles of 8 KiB
     int n_wtiles;
     const uint8_t* step_flags;
-    const float* seg_scale;
+    const float* seg_scale;      // [n_seg] in the order the clusters' last steps come
+    const uint8_t* seg_buf;      // [n_seg] accumulator of each, same order
     const float* cl_sz;
     const float* corr;           // optional [N]: sum_c s_c z_c Wsum_c[n] computed beforehand, else NULL
     const float* s_w;
@@ -275,6 +281,7 @@ cluster_gemm_kernel(const Params p)
 
     uint8_t* s_flags = smem + SL.off_flags;
     float* s_seg_scale = reinterpret_cast<float*>(smem + SL.off_seg_scale);
+    uint8_t* s_seg_buf = smem + SL.off_seg_buf;
     float* s_cl_sz = reinterpret_cast<float*>(smem + SL.off_cl_sz);
     float* s_tab = reinterpret_cast<float*>(smem + SL.off_tab);           // [2][3][TILE_N]
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SL.off_bar);
@@ -306,7 +313,7 @@ cluster_gemm_kernel(const Params p)
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     for (int i = tid; i < n_steps; i += THREADS) s_flags[i] = p.step_flags[i];
-    for (int i = tid; i < p.n_seg; i += THREADS) s_seg_scale[i] = p.seg_scale[i] * 0.0625f;   // operands were 16 * w
+    for (int i = tid; i < p.n_seg; i += THREADS) { s_seg_scale[i] = p.seg_scale[i] * 0.0625f; s_seg_buf[i] = p.seg_buf[i]; }   // operands were 16 * w
     for (int i = tid; i < p.g; i += THREADS) s_cl_sz[i] = p.cl_sz[i];
     if (warp == 1) {
         if constexpr (NCTA == 1) {
@@ -361,11 +368,11 @@ cluster_gemm_kernel(const Params p)
             // This lane is a single thread of dependent instructions, so the loop is kept short:
             // stage descriptors are built once, a K block's four step flags come as one word, and a
             // block that lies inside one cluster issues its four MMAs without any test.
-            uint32_t n_kb_done = 0, n_seg_done = 0;
+            uint32_t n_kb_done = 0;
+            uint32_t par = 0;                // bit b: parity of how many clusters accumulator b has held
             bool ok = true;
             const uint64_t a_desc0 = smem_desc_sw128(smem_base), w_desc0 = smem_desc_sw128(smem_base + A8_BYTES);
             const uint32_t* flags4 = reinterpret_cast<const uint32_t*>(s_flags);
-            uint32_t d_tmem = tmem_base;
             uint32_t f4 = flags4[0];
             for (int t = pair_id; t < p.n_tiles && ok; t += n_pairs) {
                 for (int kb = 0; kb < p.n_kb && ok; ++kb, ++n_kb_done) {
@@ -375,7 +382,9 @@ cluster_gemm_kernel(const Params p)
                     tc_fence_after();
                     // the start-address field counts 16-byte units: one stage further, 32 bytes per step
                     const uint64_t ad = a_desc0 + (uint64_t)(s * (SL.u_stage >> 4)), wd = w_desc0 + (uint64_t)(s * (SL.u_stage >> 4));
-                    if (f4 == 0) {
+                    if (f4 == 0u || f4 == 0x01010101u * STEP_BUF) {
+                        // four steps inside one cluster
+                        const uint32_t d_tmem = tmem_base + (f4 ? TILE_N : 0);
                         tc_mma_i8<NCTA>(d_tmem, ad, wd, kInstrDesc, 1u);
                         tc_mma_i8<NCTA>(d_tmem, ad + 2, wd + 2, kInstrDesc, 1u);
                         tc_mma_i8<NCTA>(d_tmem, ad + 4, wd + 4, kInstrDesc, 1u);
@@ -384,17 +393,22 @@ cluster_gemm_kernel(const Params p)
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
                             const uint32_t f = (f4 >> (8 * j)) & 0xFFu;
-                            if (f == 0) { tc_mma_i8<NCTA>(d_tmem, ad + 2 * j, wd + 2 * j, kInstrDesc, 1u); continue; }   // inside a cluster
+                            const uint32_t b = (f / STEP_BUF) & 1u;
+                            const uint32_t d_tmem = tmem_base + b * TILE_N;
+                            if ((f & (STEP_FIRST | STEP_LAST | STEP_SKIP)) == 0) {       // inside a cluster
+                                tc_mma_i8<NCTA>(d_tmem, ad + 2 * j, wd + 2 * j, kInstrDesc, 1u);
+                                continue;
+                            }
                             if (f & STEP_SKIP) continue;
                             if (f & STEP_FIRST) {
-                                if (!mbar_wait(bar(B_ACCEMPTY + (n_seg_done & 1)), ((n_seg_done >> 1) & 1) ^ 1, s_abort)) { ok = false; break; }
+                                // the accumulator's previous cluster has been drained
+                                if (!mbar_wait(bar(B_ACCEMPTY + b), ((par >> b) & 1u) ^ 1u, s_abort)) { ok = false; break; }
                                 tc_fence_after();
                             }
                             tc_mma_i8<NCTA>(d_tmem, ad + 2 * j, wd + 2 * j, kInstrDesc, (f & STEP_FIRST) ? 0u : 1u);
                             if (f & STEP_LAST) {
-                                tc_commit<NCTA>(bar(B_ACCFULL + (n_seg_done & 1)));
-                                ++n_seg_done;
-                                d_tmem = tmem_base + (n_seg_done & 1) * TILE_N;
+                                tc_commit<NCTA>(bar(B_ACCFULL + b));
+                                par ^= 1u << b;
                             }
                         }
                     }
@@ -571,7 +585,8 @@ cluster_gemm_kernel(const Params p)
         const int ew = warp - EPI_WARP0;
         const int q = ew & 3, h = ew >> 2;           // TMEM lane quarter (= warp % 4), column half
         const int et = ew * 32 + lane;               // 0..255: the column whose tile constants I prepare
-        uint32_t n_seg_done = 0, n_tile_done = 0;
+        uint32_t n_tile_done = 0;
+        uint32_t par = 0;                    // bit b: parity of how many clusters of accumulator b I have drained
         bool ok = true;
         float2 R[64];                                // running sums of columns 2 i, 2 i + 1
         for (int t = pair_id; t < p.n_tiles && ok; t += n_pairs, ++n_tile_done) {
@@ -592,9 +607,10 @@ cluster_gemm_kernel(const Params p)
             }
 #pragma unroll
             for (int i = 0; i < 64; ++i) R[i] = make_float2(0.f, 0.f);
-            for (int sgi = 0; sgi < p.n_seg; ++sgi, ++n_seg_done) {
-                const uint32_t buf = n_seg_done & 1;
-                if (!mbar_wait(bar(B_ACCFULL + buf), (n_seg_done >> 1) & 1, s_abort)) { ok = false; break; }
+            for (int sgi = 0; sgi < p.n_seg; ++sgi) {
+                const uint32_t buf = s_seg_buf[sgi];
+                if (!mbar_wait(bar(B_ACCFULL + buf), (par >> buf) & 1u, s_abort)) { ok = false; break; }
+                par ^= 1u << buf;
                 tc_fence_after();
                 const float sc = s_seg_scale[sgi];
                 const float2 sc2 = make_float2(sc, sc);
@@ -778,7 +794,7 @@ static int launch_gemm(const rptq_layout_t* Lin, const void* a_codes, int M, con
     p.n_tiles = p.tiles_m * ((N + gemm::TILE_N - 1) / gemm::TILE_N);
     p.a_codes = static_cast<const uint8_t*>(a_codes); p.a_row_bytes = Lin->row_bytes;
     p.w_codes = static_cast<const uint8_t*>(w_codes); p.n_wtiles = (int)((ld_w + 127) / 128);
-    p.step_flags = Lin->d_step_flags; p.seg_scale = Lin->d_seg_scale; p.cl_sz = Lin->d_cl_sz;
+    p.step_flags = Lin->d_step_flags; p.seg_scale = Lin->d_seg_scale; p.seg_buf = Lin->d_seg_buf; p.cl_sz = Lin->d_cl_sz;
     p.s_w = s_w; p.wsum = wsum; p.ld_w = ld_w; p.bias = static_cast<const float*>(bias);
     p.act = act; p.y_dtype = y_dtype; p.y = y; p.ldy = ldy;
     p.out_unit = Lout ? Lout->d_unit : nullptr;

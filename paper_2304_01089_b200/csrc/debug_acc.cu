@@ -17,17 +17,17 @@ __device__ __forceinline__ int dp4a_u8_s8(uint32_t a, uint32_t b, int c)
 template <int BITS>
 __global__ void debug_acc_kernel(const uint8_t* __restrict__ a_codes, int64_t a_row_bytes,
                                  const uint8_t* __restrict__ w_codes, int n_kb,
-                                 const int32_t* __restrict__ seg_off, int g, int m0, int m1, int n0, int n1,
+                                 const int32_t* __restrict__ unit_cluster, int n_units, int m0, int m1, int n0, int n1,
                                  int32_t* __restrict__ acc)
 {
     const int n = n0 + blockIdx.x * blockDim.x + threadIdx.x;
     const int m = m0 + blockIdx.y;
     const int c = blockIdx.z;
     if (n >= n1 || m >= m1) return;
-    const int step_lo = seg_off[c] / 32, step_hi = (seg_off[c + 1]) / 32;
     const uint32_t* arow = reinterpret_cast<const uint32_t*>(a_codes + (int64_t)m * a_row_bytes);
     int sum = 0;
-    for (int s = step_lo; s < step_hi; ++s) {
+    for (int s = 0; s < n_units; ++s) {
+        if (unit_cluster[s] != c) continue;      // a cluster's steps need not be adjacent
         uint32_t ap[BITS], wp[4], a8[8], w8[8];
 #pragma unroll
         for (int i = 0; i < BITS; ++i) ap[i] = arow[s * BITS + i];
@@ -56,14 +56,14 @@ extern "C" int rptq_cluster_gemm_debug_acc(const rptq_layout_t* Lin, const void*
     if (dev != Lin->device) return RPTQ_ERR_INVALID_ARG;
     if (m0 == m1 || n0 == n1) return RPTQ_OK;
     if (m1 - m0 > 65535 || Lin->g > 65535) return RPTQ_ERR_UNSUPPORTED;
-    if (!Lin->d_seg_off) return RPTQ_ERR_CUDA;
+    if (!Lin->d_unit_cluster) return RPTQ_ERR_CUDA;
     dim3 block(128), grid((n1 - n0 + 127) / 128, m1 - m0, Lin->g);
     auto st = static_cast<cudaStream_t>(stream);
     const auto* a = static_cast<const uint8_t*>(a_codes);
     const auto* w = static_cast<const uint8_t*>(w_codes);
     const int wrb = Lin->K_pad / 128;      // K blocks per row of the tile-major weight buffer
-    if (Lin->bits == 3) debug_acc_kernel<3><<<grid, block, 0, st>>>(a, Lin->row_bytes, w, wrb, Lin->d_seg_off, Lin->g, m0, m1, n0, n1, acc);
-    else if (Lin->bits == 4) debug_acc_kernel<4><<<grid, block, 0, st>>>(a, Lin->row_bytes, w, wrb, Lin->d_seg_off, Lin->g, m0, m1, n0, n1, acc);
-    else debug_acc_kernel<8><<<grid, block, 0, st>>>(a, Lin->row_bytes, w, wrb, Lin->d_seg_off, Lin->g, m0, m1, n0, n1, acc);
+    if (Lin->bits == 3) debug_acc_kernel<3><<<grid, block, 0, st>>>(a, Lin->row_bytes, w, wrb, Lin->d_unit_cluster, Lin->n_units, m0, m1, n0, n1, acc);
+    else if (Lin->bits == 4) debug_acc_kernel<4><<<grid, block, 0, st>>>(a, Lin->row_bytes, w, wrb, Lin->d_unit_cluster, Lin->n_units, m0, m1, n0, n1, acc);
+    else debug_acc_kernel<8><<<grid, block, 0, st>>>(a, Lin->row_bytes, w, wrb, Lin->d_unit_cluster, Lin->n_units, m0, m1, n0, n1, acc);
     return cudaGetLastError() == cudaSuccess ? RPTQ_OK : RPTQ_ERR_CUDA;
 }

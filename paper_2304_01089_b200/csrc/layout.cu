@@ -6,6 +6,8 @@
 #include <mutex>
 #include <new>
 
+#include <algorithm>
+
 #include "rptq_internal.h"
 
 namespace rptq {
@@ -119,11 +121,12 @@ int rptq_get_device_status(int* status)
 }
 
 int rptq_layout_create(rptq_layout_t** out, int C, int g, int bits, const int32_t* perm_host,
-                       const int32_t* cluster_size, const float* scale_host, const int32_t* zero_host)
+                       const int32_t* cluster_size, const float* scale_host, const int32_t* zero_host, int order)
 {
     if (!out) return RPTQ_ERR_INVALID_ARG;
     *out = nullptr;
     if (!perm_host || !cluster_size || !scale_host || !zero_host) return RPTQ_ERR_INVALID_ARG;
+    if (order != RPTQ_ORDER_CONTIGUOUS && order != RPTQ_ORDER_INTERLEAVED) return RPTQ_ERR_INVALID_ARG;
     if (C <= 0 || g <= 0) return RPTQ_ERR_INVALID_ARG;
     if (bits != 3 && bits != 4 && bits != 8) return RPTQ_ERR_UNSUPPORTED;
     if (C % 8 != 0 || C < 8 || C > 65528 || g > 4096) return RPTQ_ERR_UNSUPPORTED;
@@ -157,7 +160,6 @@ int rptq_layout_create(rptq_layout_t** out, int C, int g, int bits, const int32_
     L->size.assign(cluster_size, cluster_size + g);
     L->scale.assign(scale_host, scale_host + g);
     L->zero.assign(zero_host, zero_host + g);
-    L->seg_off.resize((size_t)g + 1);
     // Without a CUDA device the handle is host-only: rptq_weight_pack and rptq_layout_query work,
     // kernel launches report RPTQ_ERR_CUDA.
     int n_dev = 0;
@@ -165,32 +167,88 @@ int rptq_layout_create(rptq_layout_t** out, int C, int g, int bits, const int32_
     if (!have_device) (void)cudaGetLastError();
     if (have_device && cudaGetDevice(&L->device) != cudaSuccess) { delete L; return RPTQ_ERR_CUDA; }
 
+    // ---- unit order: a list of runs (cluster, first unit within the cluster, units)
+    struct Run { int c, u0, nu; };
+    std::vector<Run> runs;
+    std::vector<int> n_units_of((size_t)g), j_start((size_t)g);
+    {
+        int j = 0;
+        for (int c = 0; c < g; ++c) { n_units_of[c] = (cluster_size[c] + 31) / 32; j_start[c] = j; j += cluster_size[c]; }
+    }
+    constexpr int kSmallUnits = 2, kGap = 7;
+    std::vector<int> small, big;
+    for (int c = 0; c < g; ++c) {
+        if (n_units_of[c] == 0) continue;
+        (n_units_of[c] <= kSmallUnits ? small : big).push_back(c);
+    }
+    if (order == RPTQ_ORDER_INTERLEAVED && small.size() >= 2 && !big.empty()) {
+        size_t next_small = 0;
+        int since = 0;                       // larger-cluster units since the last small cluster
+        for (int c : big) {
+            int u = 0;
+            while (u < n_units_of[c]) {
+                const int take = std::min(n_units_of[c] - u, kGap - since);
+                runs.push_back({c, u, take});
+                u += take; since += take;
+                if (since == kGap) {
+                    if (next_small < small.size()) { const int t = small[next_small++]; runs.push_back({t, 0, n_units_of[t]}); }
+                    since = 0;
+                }
+            }
+        }
+        for (; next_small < small.size(); ++next_small) { const int t = small[next_small]; runs.push_back({t, 0, n_units_of[t]}); }
+    } else {
+        for (int c = 0; c < g; ++c) if (n_units_of[c] > 0) runs.push_back({c, 0, n_units_of[c]});
+    }
+
     std::vector<uint16_t> src((size_t)k_pad, (uint16_t)C);
     std::vector<UnitInfo> unit((size_t)L->n_units);
     std::vector<uint8_t> flags((size_t)L->n_units, STEP_SKIP);
     std::vector<float> seg_scale, cl_sz((size_t)g);
+    std::vector<uint8_t> seg_buf;
+    L->unit_cluster.assign((size_t)L->n_units, -1);
+    L->pos.assign((size_t)C, 0);
     for (auto& u : unit) { u.inv_s = 1.0f; u.zc = 0 - 0x4B400000; u.j0 = 0; u.nvalid = 0; }
-    int off = 0, j = 0;
-    for (int c = 0; c < g; ++c) {
-        L->seg_off[c] = off;
-        const int n = cluster_size[c];
+    for (int c = 0; c < g; ++c) cl_sz[c] = scale_host[c] * (float)zero_host[c];
+    // Accumulator of each cluster: the one that is not held by a cluster still under way; when
+    // both are free, the one whose last cluster ended longer ago (its drain has had more time).
+    int last_end[2] = {-2, -1};              // unit index at which each accumulator's last cluster ended
+    std::vector<int> buf_of((size_t)g, -1);
+    int open_buf = -1, open_cluster = -1, cur = 0;
+    for (const Run& r : runs) {
+        const int c = r.c, n = cluster_size[c];
         const float inv_s = (float)(1.0 / (double)scale_host[c]);
-        cl_sz[c] = scale_host[c] * (float)zero_host[c];
-        const int units_here = (n + 31) / 32;
-        for (int u = 0; u < units_here; ++u) {
-            UnitInfo& ui = unit[off / 32 + u];
+        for (int k = 0; k < r.nu; ++k, ++cur) {
+            const int uc = r.u0 + k;         // unit within the cluster
+            uint8_t f = 0;
+            if (uc == 0) {
+                f |= STEP_FIRST;
+                if (open_cluster >= 0 && open_cluster != c) buf_of[c] = 1 - open_buf;
+                else buf_of[c] = last_end[0] <= last_end[1] ? 0 : 1;
+                if (n_units_of[c] > r.nu) { open_cluster = c; open_buf = buf_of[c]; }   // continues in later runs
+            }
+            if (uc == n_units_of[c] - 1) {
+                f |= STEP_LAST;
+                last_end[buf_of[c]] = cur;
+                seg_scale.push_back(scale_host[c]);
+                seg_buf.push_back((uint8_t)buf_of[c]);
+                L->n_seg++;
+                if (open_cluster == c) { open_cluster = -1; open_buf = -1; }
+            }
+            if (buf_of[c]) f |= STEP_BUF;
+            flags[cur] = f;
+            L->unit_cluster[cur] = c;
+            UnitInfo& ui = unit[cur];
             ui.inv_s = inv_s;
             ui.zc = zero_host[c] - 0x4B400000;
-            ui.j0 = j + 32 * u;
-            ui.nvalid = (n - 32 * u) < 32 ? (n - 32 * u) : 32;
-            flags[off / 32 + u] = (u == 0 ? STEP_FIRST : 0) | (u == units_here - 1 ? STEP_LAST : 0);
+            ui.j0 = j_start[c] + 32 * uc;
+            ui.nvalid = (n - 32 * uc) < 32 ? (n - 32 * uc) : 32;
+            for (int e = 0; e < ui.nvalid; ++e) {
+                L->pos[ui.j0 + e] = cur * 32 + e;
+                src[cur * 32 + e] = (uint16_t)ybuf_addr(perm_host[ui.j0 + e], C);
+            }
         }
-        for (int i = 0; i < n; ++i) src[off + i] = (uint16_t)ybuf_addr(perm_host[j + i], C);
-        if (n > 0) { seg_scale.push_back(scale_host[c]); L->n_seg++; }
-        j += n;
-        off += units_here * 32;
     }
-    L->seg_off[g] = off;
 
     if (!have_device) { *out = L; return RPTQ_OK; }
     int rc = upload(&L->d_src, src.data(), src.size());
@@ -198,18 +256,19 @@ int rptq_layout_create(rptq_layout_t** out, int C, int g, int bits, const int32_
     if (rc == RPTQ_OK) rc = upload(&L->d_step_flags, flags.data(), flags.size());
     if (rc == RPTQ_OK) rc = upload(&L->d_seg_scale, seg_scale.data(), seg_scale.size());
     if (rc == RPTQ_OK) rc = upload(&L->d_cl_sz, cl_sz.data(), cl_sz.size());
-    if (rc == RPTQ_OK) rc = upload(&L->d_seg_off, L->seg_off.data(), L->seg_off.size());
+    if (rc == RPTQ_OK) rc = upload(&L->d_seg_buf, seg_buf.data(), seg_buf.size());
+    if (rc == RPTQ_OK) rc = upload(&L->d_unit_cluster, L->unit_cluster.data(), L->unit_cluster.size());
     if (rc != RPTQ_OK) { rptq_layout_destroy(L); return rc; }
     *out = L;
     return RPTQ_OK;
 }
 
-int rptq_layout_query(const rptq_layout_t* L, int* K_pad, int64_t* row_bytes, int32_t* seg_offset_out)
+int rptq_layout_query(const rptq_layout_t* L, int* K_pad, int64_t* row_bytes, int32_t* unit_cluster_out)
 {
     if (!L) return RPTQ_ERR_INVALID_ARG;
     if (K_pad) *K_pad = L->K_pad;
     if (row_bytes) *row_bytes = L->row_bytes;
-    if (seg_offset_out) std::memcpy(seg_offset_out, L->seg_off.data(), sizeof(int32_t) * ((size_t)L->g + 1));
+    if (unit_cluster_out) std::memcpy(unit_cluster_out, L->unit_cluster.data(), sizeof(int32_t) * (size_t)L->n_units);
     return RPTQ_OK;
 }
 
@@ -217,9 +276,7 @@ int rptq_layout_padded_index(const rptq_layout_t* L, int32_t* padded_index)
 {
     if (!L || !padded_index) return RPTQ_ERR_INVALID_ARG;
     for (int p = 0; p < L->K_pad; ++p) padded_index[p] = -1;
-    int j = 0;
-    for (int c = 0; c < L->g; ++c)
-        for (int i = 0; i < L->size[c]; ++i, ++j) padded_index[L->seg_off[c] + i] = L->perm[j];
+    for (int j = 0; j < L->C; ++j) padded_index[L->pos[j]] = L->perm[j];
     return RPTQ_OK;
 }
 
@@ -231,7 +288,8 @@ int rptq_layout_destroy(rptq_layout_t* L)
     cudaFree(L->d_step_flags);
     cudaFree(L->d_seg_scale);
     cudaFree(L->d_cl_sz);
-    cudaFree(L->d_seg_off);
+    cudaFree(L->d_seg_buf);
+    cudaFree(L->d_unit_cluster);
     delete L;
     return RPTQ_OK;
 }
@@ -312,13 +370,12 @@ int rptq_weight_pack(const rptq_layout_t* Lin, const float* W_host, int N, const
                 int j = 0;
                 for (int c = 0; c < g; ++c) {
                     int32_t sum = 0;
-                    uint8_t* seg = row.data() + Lin->seg_off[c];
                     for (int i = 0; i < Lin->size[c]; ++i, ++j) {
                         float q = rintf(w[Lin->perm[j]] / s);
                         q = fminf(fmaxf(q, -8.0f), 7.0f);
                         const int qi = (int)q;
                         sum += qi;
-                        seg[i] = (uint8_t)(qi & 0xF);
+                        row[Lin->pos[j]] = (uint8_t)(qi & 0xF);
                     }
                     wsum[(int64_t)c * N_pad + r] = sum;
                 }

@@ -10,8 +10,7 @@
 
 namespace rptq {
 
-// One entry per group of 32 padded positions ("unit"). A unit never straddles two clusters
-// because every cluster segment starts at a multiple of 32.
+// One entry per group of 32 padded positions ("unit"). A unit belongs to one cluster.
 struct UnitInfo {
     float inv_s;      // (float)(1.0 / (double)s_c)
     int32_t zc;       // z_c - 0x4B400000: added to the bit pattern of (t + 1.5*2^23)
@@ -21,7 +20,9 @@ struct UnitInfo {
 static_assert(sizeof(UnitInfo) == 16, "UnitInfo is loaded as one 16-byte vector");
 
 // Flags of one contraction step (32 consecutive padded positions) along K.
-enum : uint8_t { STEP_FIRST = 1, STEP_LAST = 2, STEP_SKIP = 4 };
+// FIRST / LAST: first / last step of its cluster (a cluster's steps need not be adjacent); SKIP: no
+// cluster; BUF: which of the two accumulators the cluster uses.
+enum : uint8_t { STEP_FIRST = 1, STEP_LAST = 2, STEP_SKIP = 4, STEP_BUF = 8 };
 
 constexpr int kMaxGemmSegments = 1024;
 
@@ -40,15 +41,18 @@ struct rptq_layout {
     int64_t row_bytes = 0;
     int n_units = 0;   // K_pad / 32
     int n_seg = 0;     // clusters with n_c > 0
-    std::vector<int32_t> perm, size, seg_off, zero;
+    std::vector<int32_t> perm, size, zero;
+    std::vector<int32_t> pos;            // [C]       padded position of reordered channel j
+    std::vector<int32_t> unit_cluster;   // [n_units] owning cluster, -1 past the last cluster
     std::vector<float> scale;
     // device tables
     uint16_t* d_src = nullptr;          // [K_pad] ybuf_addr of each padded position's channel, C = pad
     rptq::UnitInfo* d_unit = nullptr;   // [n_units]
     uint8_t* d_step_flags = nullptr;    // [n_units]
-    float* d_seg_scale = nullptr;       // [n_seg]  s_c of the non-empty clusters, in K order
+    float* d_seg_scale = nullptr;       // [n_seg]  s_c of the non-empty clusters, in the order their last steps come
+    uint8_t* d_seg_buf = nullptr;       // [n_seg]  the accumulator each of them uses, same order
     float* d_cl_sz = nullptr;           // [g]      s_c * z_c
-    int32_t* d_seg_off = nullptr;       // [g+1]    padded segment offsets
+    int32_t* d_unit_cluster = nullptr;  // [n_units]
 };
 
 namespace rptq {

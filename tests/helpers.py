@@ -17,9 +17,9 @@ class Site:
         self.draws = workloads.kmeans_draws(w, 0, self.g)
         self.cal = calibration.calibrate(x_cal, self.gamma, self.beta, self.g, self.bits, self.draws)
 
-    def layout(self):
+    def layout(self, order=0):
         from paper_2304_01089_b200 import binding
-        return binding.Layout(self.cal.perm, self.cal.size, self.cal.scale, self.cal.zero, self.bits)
+        return binding.Layout(self.cal.perm, self.cal.size, self.cal.scale, self.cal.zero, self.bits, order=order)
 
 
 def random_layout_params(rng, C, g, bits, allow_empty=True):

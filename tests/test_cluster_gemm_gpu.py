@@ -28,14 +28,17 @@ def _case(rng, M, N, C, g, bits, n_pad=None, allow_empty=True):
                 a=a, k_pad=k_pad, bits=bits, M=M, N=N, n_pad=n_pad)
 
 
-def _dev(case):
+def _dev(case, order=0):
+    """Device inputs of a case. The oracle's arrays are in the contiguous unit order; their columns
+    are moved to the layout's own order before packing."""
     import torch
     from paper_2304_01089_b200 import binding
-    L = binding.Layout(case["perm"], case["size"], case["scale"], case["zero"], case["bits"])
+    L = binding.Layout(case["perm"], case["size"], case["scale"], case["zero"], case["bits"], order=order)
     assert L.K_pad == case["k_pad"]
+    m = L.contiguous_position()
     d = dict(L=L,
-             a=torch.from_numpy(oracle.pack(case["a"], case["bits"])).cuda(),
-             w=torch.from_numpy(oracle.pack_weights(case["w_codes"])).cuda(),
+             a=torch.from_numpy(oracle.pack(np.ascontiguousarray(case["a"][:, m]), case["bits"])).cuda(),
+             w=torch.from_numpy(oracle.pack_weights(np.ascontiguousarray(case["w_codes"][:, m]))).cuda(),
              s_w=torch.from_numpy(case["s_w"]).cuda(),
              wsum=torch.from_numpy(case["wsum"]).cuda())
     return d
@@ -125,6 +128,50 @@ def test_small_and_ragged_shapes(bits, M, N, C, g):
     want_b = _oracle_y(case, bias=bias[:N], relu=True)
     assert np.max(np.abs(yb - want_b)) <= TOL * np.abs(want).max()
     assert yb.min() >= 0.0
+
+
+@pytest.mark.parametrize("bits,M", [(3, 300), (4, 100), (8, 257)])
+def test_interleaved_unit_order(bits, M):
+    """Many one- and two-unit clusters among a few large ones, as calibration produces them: the
+    interleaved layout gives the oracle's result, and each cluster's accumulator bit for bit."""
+    import torch
+    from paper_2304_01089_b200 import binding
+    rng = np.random.default_rng(900 + bits)
+    size = np.array([1, 1, 2, 3, 9, 13, 0, 40, 5, 53, 173, 434, 530, 7, 64, 33, 664, 300, 2, 1, 1, 6], np.int32)
+    size[-1] += (-int(size.sum())) % 8
+    C, g, N = int(size.sum()), len(size), 520
+    perm = rng.permutation(C).astype(np.int32)
+    scale = rng.uniform(0.05, 1.5, size=g).astype(np.float32)
+    zero = rng.integers(0, 1 << bits, size=g).astype(np.int32)
+    W = (rng.normal(size=(N, C)) * 0.02).astype(np.float32)
+    w_codes, s_w, wsum = oracle.weight_quantize(W, perm, size, None, N)
+    off, k_pad = oracle.segment_offsets(size)
+    a = np.zeros((M, k_pad), np.uint8)
+    for c in range(g):
+        a[:, off[c]:off[c] + size[c]] = rng.integers(0, 1 << bits, size=(M, size[c]))
+    case = dict(perm=perm, size=size, scale=scale, zero=zero, w_codes=w_codes, s_w=s_w, wsum=wsum,
+                a=a, k_pad=k_pad, bits=bits, M=M, N=N, n_pad=N)
+    d = _dev(case, order=binding.ORDER_INTERLEAVED)
+    assert not np.array_equal(d["L"].contiguous_position(), np.arange(k_pad))
+    want = _oracle_y(case)
+    y = _gemm(case, d)
+    assert np.max(np.abs(y - want)) <= TOL * np.abs(want).max()
+    y_contig = _gemm(case, _dev(case))
+    assert np.max(np.abs(y - y_contig)) <= 1e-5 * np.abs(want).max()      # same sums, another order
+    acc = torch.full((g, M, N), -1, dtype=torch.int32, device="cuda")
+    binding.cluster_gemm_debug_acc(d["L"], d["a"], M, d["w"], N, 0, M, 0, N, acc)
+    torch.cuda.synchronize()
+    assert np.array_equal(acc.cpu().numpy().astype(np.int64), oracle.cluster_acc(a, w_codes, size))
+    # one cluster at a time through the tensor-core path (scale 1 for it, vanishing for the others)
+    ones = torch.ones(N, dtype=torch.float32, device="cuda")
+    zeros_ws = torch.zeros_like(d["wsum"])
+    want_acc = oracle.cluster_acc(a, w_codes, size)
+    for c in (0, 3, 7, 11, 12, 16, 21):
+        sc = np.full(g, 2.0 ** -80, np.float32)
+        sc[c] = 1.0
+        L1 = binding.Layout(perm, size, sc, np.zeros(g, np.int32), bits, order=binding.ORDER_INTERLEAVED)
+        y1 = _gemm(case, d, s_w=ones, wsum=zeros_ws, L=L1)
+        assert np.array_equal(y1.astype(np.int64), want_acc[c]), f"cluster {c}"
 
 
 def test_two_launches_on_two_streams_give_identical_bytes():

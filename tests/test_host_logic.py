@@ -41,7 +41,12 @@ def test_layout_validation_and_padded_offsets(binding):
     perm, size, scale, zero = random_layout_params(rng, C, g, bits)
     L = binding.Layout(perm, size, scale, zero, bits)
     off, k_pad = oracle.segment_offsets(size)
-    assert L.K_pad == k_pad and np.array_equal(L.seg_off, off) and L.row_bytes == k_pad // 2
+    assert L.K_pad == k_pad and L.row_bytes == k_pad // 2
+    want_uc = np.full(k_pad // 32, -1, np.int32)
+    for c in range(g):
+        want_uc[off[c] // 32:off[c + 1] // 32] = c
+    assert np.array_equal(L.unit_cluster, want_uc)
+    assert np.array_equal(L.contiguous_position(), np.arange(k_pad))
     off2, k_pad2 = calibration.segment_offsets(size)
     assert k_pad2 == k_pad and np.array_equal(off2, off)
     bad = perm.copy(); bad[3] = bad[4]
@@ -102,6 +107,61 @@ def test_weight_pack_matches_the_oracle_bit_for_bit(binding):
         want[off[c]:off[c] + size[c]] = perm[j:j + size[c]]
         j += size[c]
     assert np.array_equal(idx, want)
+
+
+def test_interleaved_unit_order(binding):
+    """Small clusters are placed between the units of the larger ones; every channel keeps its
+    cluster and its order within the cluster; packed weights follow the same order."""
+    rng = np.random.default_rng(5)
+    size = np.array([1, 2, 33, 700, 0, 5, 64, 300, 40, 200, 7, 3, 133], np.int32)
+    C, g, bits = int(size.sum()), len(size), 3
+    assert C % 8 == 0
+    perm = rng.permutation(C).astype(np.int32)
+    scale = rng.uniform(0.05, 1.5, size=g).astype(np.float32)
+    zero = rng.integers(0, 8, size=g).astype(np.int32)
+    Lc = binding.Layout(perm, size, scale, zero, bits)
+    Li = binding.Layout(perm, size, scale, zero, bits, order=binding.ORDER_INTERLEAVED)
+    assert Li.K_pad == Lc.K_pad and Li.row_bytes == Lc.row_bytes
+    units = (size + 31) // 32
+    uc = Li.unit_cluster
+    assert np.array_equal(np.bincount(uc[uc >= 0], minlength=g), units)
+    assert np.all(uc[int(units.sum()):] == -1)
+    # clusters of one or two units come after every seven units of larger clusters, each in one piece
+    small = [c for c in range(g) if 1 <= units[c] <= 2]
+    big_run, placed = 0, []
+    u = 0
+    while u < int(units.sum()):
+        c = int(uc[u])
+        if c in small:
+            assert np.all(uc[u:u + units[c]] == c)
+            placed.append((c, big_run))
+            big_run = 0
+            u += int(units[c])
+        else:
+            big_run += 1
+            u += 1
+    assert [c for c, _ in placed] == small
+    n_big_units = int(units.sum()) - sum(int(units[c]) for c in small)
+    assert all(run == 7 for _, run in placed[:n_big_units // 7])
+    # larger clusters keep their relative order and the order of their own units
+    firsts = [int(np.argmax(uc == c)) for c in range(g) if units[c] > 2]
+    assert firsts == sorted(firsts)
+    # every channel sits in a unit of its cluster, in the order of S
+    idx_c, idx_i, m = Lc.padded_index(), Li.padded_index(), Li.contiguous_position()
+    assert np.array_equal(idx_i, idx_c[m])
+    assert sorted(idx_i[idx_i >= 0].tolist()) == list(range(C))
+    # packed weights: the oracle's codes with their columns moved to this order
+    W = rng.normal(size=(70, C)).astype(np.float32)
+    packed, s_w, wsum = binding.weight_pack(Li, W, None, 72)
+    w_codes, s_w_o, wsum_o = oracle.weight_quantize(W, perm, size, None, 72)
+    assert np.array_equal(packed, oracle.pack_weights(np.ascontiguousarray(w_codes[:, m])))
+    assert np.array_equal(s_w, s_w_o) and np.array_equal(wsum, wsum_o)
+    # fewer than two small clusters: nothing to interleave
+    size2 = np.array([100, 60, 96], np.int32)
+    L2 = binding.Layout(rng.permutation(256).astype(np.int32), size2, scale[:3], zero[:3], 4, order=binding.ORDER_INTERLEAVED)
+    assert np.array_equal(L2.contiguous_position(), np.arange(L2.K_pad))
+    with pytest.raises(binding.RptqError):
+        binding.Layout(perm, size, scale, zero, bits, order=2)
 
 
 def test_numpy_calibration_agrees_with_the_oracle_calibration():

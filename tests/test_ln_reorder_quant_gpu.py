@@ -36,14 +36,17 @@ def _run(layout, x16, gamma16, beta16, want_y=True, ldx=None, stream=None):
     return codes_h[:M], y_h
 
 
-def _check_against_oracle(x16, gamma16, beta16, perm, size, scale32, zero, bits, packed, y_dbg, full_rate=0.9999):
+def _check_against_oracle(x16, gamma16, beta16, perm, size, scale32, zero, bits, packed, y_dbg, full_rate=0.9999, pos=None):
+    """`pos`: the layout's contiguous_position() when its unit order is not the contiguous one (the
+    oracle's codes are in contiguous order)."""
     M, C = x16.shape
     _, k_pad = oracle.segment_offsets(size)
-    got = oracle.unpack(packed, k_pad, bits)
+    pos = np.arange(k_pad) if pos is None else pos
+    got = oracle.unpack(packed, k_pad, bits)[:, np.argsort(pos)]          # back to contiguous order
     # (1) the decision, bit for bit, from the kernel's own fp32 LayerNorm outputs
     want32 = oracle.quantize_f32(y_dbg, size, scale32, zero, bits)
     assert np.array_equal(got, want32), "codes differ from the fp32-decision oracle on identical LN outputs"
-    assert np.array_equal(packed, oracle.pack(want32, bits)), "packed bytes differ from the documented format"
+    assert np.array_equal(packed, oracle.pack(np.ascontiguousarray(want32[:, pos]), bits)), "packed bytes differ from the documented format"
     # (2) the whole step against the fp64 oracle
     y64 = oracle.reorder(oracle.layernorm(x16, gamma16, beta16, EPS), perm)
     want64 = oracle.quantize(y64, size, scale32.astype(np.float64), zero, bits)
@@ -61,11 +64,12 @@ def _check_against_oracle(x16, gamma16, beta16, perm, size, scale32, zero, bits,
 
 @pytest.mark.parametrize("name", ["opt-125m", "opt-1.3b", "opt-6.7b", "opt-66b", "opt-175b"])
 def test_workload_configs_full_size(name):
+    from paper_2304_01089_b200 import binding
     site = Site(workloads.WORKLOADS[name])
-    L = site.layout()
+    L = site.layout(order=binding.ORDER_INTERLEAVED)       # the order the benchmark uses
     packed, y_dbg = _run(L, site.x, site.gamma, site.beta)
     rate = _check_against_oracle(site.x, site.gamma, site.beta, site.cal.perm, site.cal.size, site.cal.scale,
-                                 site.cal.zero, site.bits, packed, y_dbg)
+                                 site.cal.zero, site.bits, packed, y_dbg, pos=L.contiguous_position())
     print(f"{name}: {rate:.6f} of codes equal the fp64 oracle")
     # same launch without the debug output and on another stream: identical bytes
     import torch

@@ -35,7 +35,9 @@ def _pack_weights_both(L, site_w, li, n_out, hidden, out_perm=None, n_pad=None):
     w_codes_o, s_w_o, wsum_o = oracle.weight_quantize(W, L._perm, L._size, out_perm, n_pad)
     packed, s_w, wsum = binding.weight_pack(L, W, out_perm, n_pad)
     del W
-    assert np.array_equal(packed, oracle.pack_weights(w_codes_o)), "packed weights differ from the oracle's"
+    in_lib_order = np.ascontiguousarray(w_codes_o[:, L.contiguous_position()])
+    assert np.array_equal(packed, oracle.pack_weights(in_lib_order)), "packed weights differ from the oracle's"
+    del in_lib_order
     assert np.array_equal(s_w, s_w_o) and np.array_equal(wsum, wsum_o)
     dev = dict(w=torch.from_numpy(packed).cuda(), s_w=torch.from_numpy(s_w).cuda(), wsum=torch.from_numpy(wsum).cuda())
     return dev, w_codes_o, s_w_o, wsum_o
@@ -43,7 +45,8 @@ def _pack_weights_both(L, site_w, li, n_out, hidden, out_perm=None, n_pad=None):
 
 def _ln_codes(site, L, M):
     """Kernel (a) on the first M test tokens; returns the device code buffer and the oracle's codes
-    for the sampled rows (which replace the kernel's in the buffer)."""
+    for the sampled rows (which replace the kernel's in the buffer). The oracle's codes are in the
+    contiguous unit order; `pos` moves them to the layout's."""
     import torch
     from paper_2304_01089_b200 import binding
     x = site.x[:M]
@@ -54,10 +57,12 @@ def _ln_codes(site, L, M):
     rows = _sample_rows(M)
     y64 = oracle.reorder(oracle.layernorm(x[rows], site.gamma, site.beta, EPS), site.cal.perm)
     want = oracle.quantize(y64, site.cal.size, site.cal.scale.astype(np.float64), site.cal.zero, site.bits)
+    pos = L.contiguous_position()
+    want_lib = np.ascontiguousarray(want[:, pos])
     got = oracle.unpack(codes[torch.from_numpy(rows).cuda()].cpu().numpy(), L.K_pad, site.bits)
-    diff = np.abs(got.astype(int) - want.astype(int))
+    diff = np.abs(got.astype(int) - want_lib.astype(int))
     assert diff.max() <= 1 and (diff != 0).mean() <= 1e-4 * (L.K_pad / site.w.hidden) + 2e-4
-    codes[torch.from_numpy(rows).cuda()] = torch.from_numpy(oracle.pack(want, site.bits)).cuda()
+    codes[torch.from_numpy(rows).cuda()] = torch.from_numpy(oracle.pack(want_lib, site.bits)).cuda()
     return codes, rows, want
 
 
@@ -67,7 +72,7 @@ def test_layernorm_to_linear_full_size(name, li, Ms):
     from paper_2304_01089_b200 import binding
     site = Site(workloads.WORKLOADS[name])
     w = site.w
-    L = site.layout()
+    L = site.layout(order=binding.ORDER_INTERLEAVED)
     n_out = w.linears[li].n_out
     dev, w_codes_o, s_w_o, wsum_o = _pack_weights_both(L, w, li, n_out, w.hidden)
     bias = workloads.bias_vector(w, li, n_out)
@@ -109,7 +114,7 @@ def test_fc1_relu_requantise_fc2_chain_full_size():
     w = site.w
     M, C, H = w.tokens, w.hidden, w.linears[0].n_out
     g2, bits2 = w.chain_clusters, w.bits
-    L1 = site.layout()
+    L1 = site.layout(order=binding.ORDER_INTERLEAVED)
     b1 = workloads.bias_vector(w, 0, H)
 
     # --- calibrate the FC1-output site from the product path itself on the calibration tokens
@@ -125,9 +130,13 @@ def test_fc1_relu_requantise_fc2_chain_full_size():
     h_min, h_max = h_cal.amin(0).cpu().numpy().astype(np.float64), h_cal.amax(0).cpu().numpy().astype(np.float64)
     del h_cal, cal_codes, dev1_id, w1_o_id
     cal2 = calibration.calibrate_from_minmax(h_min, h_max, g2, bits2, workloads.kmeans_draws(w, 1, g2))
-    L2 = binding.Layout(cal2.perm, cal2.size, cal2.scale, cal2.zero, bits2)
-    idx = L2.padded_index()
+    L2 = binding.Layout(cal2.perm, cal2.size, cal2.scale, cal2.zero, bits2, order=binding.ORDER_INTERLEAVED)
+    idx = L2.padded_index()          # original hidden channel at each position of the second site's rows
     K2 = L2.K_pad
+    pos2 = L2.contiguous_position()
+    where = np.empty(H, np.int64)    # position of each hidden channel in the second site's rows
+    where[idx[idx >= 0]] = np.nonzero(idx >= 0)[0]
+    in_S_order = where[cal2.perm]    # ... of the channels in the order of the reorder index
     print(f"FC1-output site: K_pad {K2}, cluster sizes {sorted(cal2.size.tolist())[:8]} ... {sorted(cal2.size.tolist())[-4:]}")
 
     # --- FC1 with its rows in the next site's padded order, FC2 on that site's codes
@@ -146,14 +155,15 @@ def test_fc1_relu_requantise_fc2_chain_full_size():
     h64 = oracle.cluster_gemm(a_rows, w1_o, site.cal.size, site.cal.scale.astype(np.float64), site.cal.zero, s1_o, ws1_o,
                               bias=b1p, relu=True)
     real = idx >= 0
-    want2 = oracle.quantize(h64[:, real], cal2.size, cal2.scale.astype(np.float64), cal2.zero, bits2)
+    want2 = oracle.quantize(h64[:, in_S_order], cal2.size, cal2.scale.astype(np.float64), cal2.zero, bits2)
+    want2_lib = np.ascontiguousarray(want2[:, pos2])
     got2 = oracle.unpack(h_codes[ridx].cpu().numpy(), K2, bits2)
-    diff = np.abs(got2.astype(int) - want2.astype(int))
+    diff = np.abs(got2.astype(int) - want2_lib.astype(int))
     print(f"re-quantised FC1 output: {(diff != 0).mean():.2e} of codes differ from the fp64 oracle, max {diff.max()}")
     assert diff.max() <= 1 and (diff != 0).mean() <= 3e-4
     assert not got2[:, ~real].any()
     # FC2 at full size with the oracle's codes planted in the sampled rows
-    h_codes[ridx] = torch.from_numpy(oracle.pack(want2, bits2)).cuda()
+    h_codes[ridx] = torch.from_numpy(oracle.pack(want2_lib, bits2)).cuda()
     y = torch.full((M, C), float("nan"), dtype=torch.float32, device="cuda")
     binding.cluster_gemm(L2, h_codes, M, dev2["w"], dev2["s_w"], dev2["wsum"], C, y)
     torch.cuda.synchronize()
