@@ -368,20 +368,24 @@ cluster_gemm_kernel(const Params p)
             // This lane is a single thread of dependent instructions, so the loop is kept short:
             // stage descriptors are built once, a K block's four step flags come as one word, and a
             // block that lies inside one cluster issues its four MMAs without any test.
-            uint32_t n_kb_done = 0;
+            // (the loop runs over all K blocks of all of this pair's tiles with one counter: the
+            // lane has few registers)
             uint32_t par = 0;                // bit b: parity of how many clusters accumulator b has held
             bool ok = true;
-            const uint64_t a_desc0 = smem_desc_sw128(smem_base), w_desc0 = smem_desc_sw128(smem_base + A8_BYTES);
+            const uint64_t a_desc0 = smem_desc_sw128(smem_base);
             const uint32_t* flags4 = reinterpret_cast<const uint32_t*>(s_flags);
             uint32_t f4 = flags4[0];
-            for (int t = pair_id; t < p.n_tiles && ok; t += n_pairs) {
-                for (int kb = 0; kb < p.n_kb && ok; ++kb, ++n_kb_done) {
+            const uint32_t total_kb = (uint32_t)(((p.n_tiles - pair_id + n_pairs - 1) / n_pairs) * p.n_kb);
+            int kb = 0;
+            for (uint32_t n_kb_done = 0; n_kb_done < total_kb; ++n_kb_done) {
                     const int s = n_kb_done % N_U;
-                    const uint32_t f4_next = flags4[kb + 1 < p.n_kb ? kb + 1 : 0];    // read while waiting
+                    kb = kb + 1 == p.n_kb ? 0 : kb + 1;
+                    const uint32_t f4_next = flags4[kb];                              // read while waiting
                     if (!mbar_wait(bar(B_UFULL + s), (n_kb_done / N_U) & 1, s_abort)) { ok = false; break; }
                     tc_fence_after();
-                    // the start-address field counts 16-byte units: one stage further, 32 bytes per step
-                    const uint64_t ad = a_desc0 + (uint64_t)(s * (SL.u_stage >> 4)), wd = w_desc0 + (uint64_t)(s * (SL.u_stage >> 4));
+                    // the start-address field counts 16-byte units: one stage further, 32 bytes per step;
+                    // the weight operand follows the activation operand in the stage
+                    const uint64_t ad = a_desc0 + (uint64_t)(s * (SL.u_stage >> 4)), wd = ad + (uint64_t)(A8_BYTES >> 4);
                     if (f4 == 0u || f4 == 0x01010101u * STEP_BUF) {
                         // four steps inside one cluster
                         const uint32_t d_tmem = tmem_base + (f4 ? TILE_N : 0);
@@ -411,10 +415,10 @@ cluster_gemm_kernel(const Params p)
                                 par ^= 1u << b;
                             }
                         }
+                        if (!ok) break;
                     }
                     tc_commit<NCTA>(bar(B_UEMPTY + s));      // the stage may be overwritten once these MMAs have read it
                     f4 = f4_next;
-                }
             }
             if (!ok) {
                 tc_commit<NCTA>(bar(B_DRAIN));
