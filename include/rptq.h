@@ -27,13 +27,15 @@
  *
  * Padded layout (not in the paper; the tensor-core contraction step is 32 codes wide and operands
  * are staged in blocks of 128): a row of codes is K_pad/32 units of 32 positions. Cluster c owns
- * roundup32(n_c)/32 units; its channels fill them in the order of S, so only its last unit can
- * hold pad positions (at the end). K_pad = max(128, roundup128(sum_c roundup32(n_c))); the units
+ * roundup32(n_c)/32 units, filled in order, so only its last unit can hold pad positions (at the
+ * end). WHICH channel of the cluster sits at which of the cluster's positions is the library's
+ * choice (all of them share s_c and z_c; the choice spreads a warp's shared-memory reads in
+ * rptq_ln_reorder_quant over the banks): rptq_layout_padded_index reports it. K_pad = max(128, roundup128(sum_c roundup32(n_c))); the units
  * left over at the end of the row belong to no cluster. Pad positions hold activation code 0 and
  * weight code 0. Two unit orders:
  *   RPTQ_ORDER_CONTIGUOUS   the clusters' units follow one another in the order of S, so cluster
- *                           c occupies positions seg_off[c] .. seg_off[c] + n_c - 1 with
- *                           seg_off[c] = sum_{c' < c} roundup32(n_c');
+ *                           c occupies n_c of the positions seg_off[c] .. seg_off[c] + roundup32(n_c) - 1
+ *                           with seg_off[c] = sum_{c' < c} roundup32(n_c');
  *   RPTQ_ORDER_INTERLEAVED  clusters of one or two units are placed between the units of the
  *                           larger clusters, one after every seven larger-cluster units (those left
  *                           over follow at the end); a larger cluster's units keep their order

@@ -137,21 +137,30 @@ class Layout:
 
     def contiguous_position(self) -> np.ndarray:
         """int32 [K_pad]: for each position of this layout, the position that holds the same channel
-        (or pad) in the contiguous unit order, where cluster c starts at sum_{c' < c} roundup32(n_c').
-        A [*, K_pad] array `a` in contiguous order becomes `a[:, m]` in this layout's order."""
-        units = (self._size.astype(np.int64) + 31) // 32
-        first = np.concatenate([[0], np.cumsum(units)])
-        seen = np.zeros(self.g, np.int64)
-        tail = int(first[-1])
+        (or a pad of the same cluster) in the plain contiguous order, where cluster c starts at
+        seg_off[c] = sum_{c' < c} roundup32(n_c') and holds its channels in the order of S.
+        A [*, K_pad] array `a` in that order becomes `a[:, m]` in this layout's order."""
+        size = self._size.astype(np.int64)
+        seg_off = np.concatenate([[0], np.cumsum((size + 31) // 32 * 32)])
+        j_start = np.concatenate([[0], np.cumsum(size)])
+        plain = np.empty(self.C, np.int64)               # plain[ch]: contiguous position of channel ch
+        for c in range(self.g):
+            plain[self._perm[j_start[c]:j_start[c + 1]]] = seg_off[c] + np.arange(size[c])
+        idx = self.padded_index()
         out = np.empty(self.K_pad, np.int32)
-        for u, c in enumerate(self.unit_cluster):
+        next_pad = (seg_off[:-1] + size).copy()          # first pad position of each cluster
+        tail = int(seg_off[-1])
+        for p in range(self.K_pad):
+            if idx[p] >= 0:
+                out[p] = plain[idx[p]]
+                continue
+            c = self.unit_cluster[p // 32]
             if c < 0:
-                cu = tail
+                out[p] = tail
                 tail += 1
             else:
-                cu = int(first[c] + seen[c])
-                seen[c] += 1
-            out[32 * u:32 * u + 32] = np.arange(32 * cu, 32 * cu + 32)
+                out[p] = next_pad[c]
+                next_pad[c] += 1
         return out
 
     def destroy(self) -> None:

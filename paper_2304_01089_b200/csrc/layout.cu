@@ -201,7 +201,8 @@ int rptq_layout_create(rptq_layout_t** out, int C, int g, int bits, const int32_
         for (int c = 0; c < g; ++c) if (n_units_of[c] > 0) runs.push_back({c, 0, n_units_of[c]});
     }
 
-    std::vector<uint16_t> src((size_t)k_pad, (uint16_t)C);
+    std::vector<uint16_t> src((size_t)k_pad, (uint16_t)C);       // channel at each position, C at pads
+    std::vector<int32_t> jidx((size_t)k_pad, -1);                // reordered index at each position, -1 at pads
     std::vector<UnitInfo> unit((size_t)L->n_units);
     std::vector<uint8_t> flags((size_t)L->n_units, STEP_SKIP);
     std::vector<float> seg_scale, cl_sz((size_t)g);
@@ -243,15 +244,49 @@ int rptq_layout_create(rptq_layout_t** out, int C, int g, int bits, const int32_
             ui.zc = zero_host[c] - 0x4B400000;
             ui.j0 = j_start[c] + 32 * uc;
             ui.nvalid = (n - 32 * uc) < 32 ? (n - 32 * uc) : 32;
-            for (int e = 0; e < ui.nvalid; ++e) {
-                L->pos[ui.j0 + e] = cur * 32 + e;
-                src[cur * 32 + e] = (uint16_t)ybuf_addr(perm_host[ui.j0 + e], C);
-            }
         }
+    }
+    // ---- which channel of a cluster goes to which of the cluster's positions. All channels of a
+    // cluster share (s_c, z_c), so any assignment is the same quantisation. rptq_ln_reorder_quant
+    // gives every unit to one thread, and the 32 threads of a warp (32 consecutive units) read
+    // element e of their units in the same instruction, from the raw fp16 row in shared memory:
+    // channel ch sits in bank (ch / 2) mod 32. Rows of 32 such reads are filled greedily with
+    // channels from 32 different banks, always from the fullest bank of the lane's cluster.
+    {
+        std::vector<std::vector<int>> pool((size_t)g * 32);          // [cluster][bank]: reordered indices j, descending
+        for (int c = 0; c < g; ++c)
+            for (int i = cluster_size[c] - 1; i >= 0; --i) {
+                const int j = j_start[c] + i;
+                pool[(size_t)c * 32 + ((perm_host[j] >> 1) & 31)].push_back(j);
+            }
+        for (int w0 = 0; w0 < L->n_units; w0 += 32)
+            for (int e = 0; e < 32; ++e) {
+                uint32_t used = 0;
+                for (int l = 0; l < 32 && w0 + l < L->n_units; ++l) {
+                    const int u = w0 + l, c = L->unit_cluster[u];
+                    if (c < 0 || e >= unit[u].nvalid) continue;
+                    int best = -1, any = -1;
+                    size_t best_n = 0, any_n = 0;
+                    for (int b = 0; b < 32; ++b) {
+                        const size_t n_b = pool[(size_t)c * 32 + b].size();
+                        if (n_b > any_n) { any_n = n_b; any = b; }
+                        if (!((used >> b) & 1u) && n_b > best_n) { best_n = n_b; best = b; }
+                    }
+                    const int b = best >= 0 ? best : any;
+                    std::vector<int>& from = pool[(size_t)c * 32 + b];
+                    const int j = from.back();
+                    from.pop_back();
+                    used |= 1u << b;
+                    L->pos[j] = u * 32 + e;
+                    src[u * 32 + e] = (uint16_t)perm_host[j];
+                    jidx[u * 32 + e] = j;
+                }
+            }
     }
 
     if (!have_device) { *out = L; return RPTQ_OK; }
     int rc = upload(&L->d_src, src.data(), src.size());
+    if (rc == RPTQ_OK) rc = upload(&L->d_jidx, jidx.data(), jidx.size());
     if (rc == RPTQ_OK) rc = upload(&L->d_unit, unit.data(), unit.size());
     if (rc == RPTQ_OK) rc = upload(&L->d_step_flags, flags.data(), flags.size());
     if (rc == RPTQ_OK) rc = upload(&L->d_seg_scale, seg_scale.data(), seg_scale.size());
@@ -284,6 +319,7 @@ int rptq_layout_destroy(rptq_layout_t* L)
 {
     if (!L) return RPTQ_OK;
     cudaFree(L->d_src);
+    cudaFree(L->d_jidx);
     cudaFree(L->d_unit);
     cudaFree(L->d_step_flags);
     cudaFree(L->d_seg_scale);

@@ -2,15 +2,16 @@
 // per-cluster quantiser (Eq. 1 applied per cluster, Appendix) and packed stores.
 //
 // The paper scatters on write ("the write address is additionally offset based on the reorder
-// index"). Packed sub-byte codes need whole words written at once, so here the row is normalised
-// into shared memory in channel order and every thread gathers the 32 channels of one output
-// unit (32 consecutive padded positions, always inside one cluster), quantises them with that
-// cluster's parameters held in registers, and stores 12/16/32 contiguous bytes.
+// index"). Packed sub-byte codes need whole words written at once, so here every thread gathers the
+// 32 channels of one output unit (32 consecutive padded positions, always inside one cluster)
+// straight from the raw fp16 row in shared memory, normalises them with the row's statistics and
+// its own channels' gains and biases (held in registers across rows), quantises them with the
+// cluster's parameters and stores 12/16/32 contiguous bytes.
 //
-// Memory-bound by design. A block is persistent over rows; rows arrive through a ring of
-// shared-memory slots filled by the copy engine several rows ahead; the shared-memory addresses
-// of a thread's 32 source channels and its unit's parameters stay in registers across rows; the
-// LayerNorm arithmetic uses the packed two-wide fp32 instructions of sm_100.
+// Memory-bound by design. A block is persistent over rows. Rows arrive through a ring of
+// shared-memory slots that the copy engine fills many rows ahead; a few warps compute each row's
+// mean and variance (one warp per row, no block-wide barrier); the gather warps follow. The
+// hand-offs are mbarriers per ring slot: landed -> statistics ready -> slot free.
 #include <cuda_fp16.h>
 
 #include <mutex>
@@ -51,21 +52,6 @@ __device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c)
     return d;
 }
 
-__device__ __forceinline__ float lds_f32(uint32_t addr)
-{
-    float v;
-    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
-    return v;
-}
-
-__device__ __forceinline__ void bar_sync(int id, int count) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory"); }
-__device__ __forceinline__ void bar_arrive(int id, int count) { asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(count) : "memory"); }
-__device__ __forceinline__ uint4 lds_v4(uint32_t addr)
-{
-    uint4 v;
-    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
-    return v;
-}
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 {
     uint32_t ok;
@@ -76,226 +62,213 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+constexpr long long kLnWaitBudgetCycles = 4000000000ll;   // about two seconds at the SM clock
 
-// The block is split into two groups of warps that work on consecutive rows at the same time:
-//   LN warps      (TL threads)  take a row from a shared-memory ring that the copy engine fills
-//                               several rows ahead (one contiguous cp.async.bulk per row: at 18-24 KB
-//                               a row, one row in flight per SM would leave HBM idle most of the
-//                               time), reduce mean and variance, and normalise the row into one of
-//                               two shared-memory buffers in channel order
-//   gather warps  (TG threads)  each thread owns one output unit (32 consecutive padded positions,
-//                               always inside one cluster): it reads its 32 source channels from the
-//                               buffer, quantises with the cluster's parameters and stores 12/16/32
-//                               contiguous bytes
-// so the reductions of row i+1 overlap the gather of row i. Named barriers hand the buffers over.
-// The only wait on the copy engine is bounded: if it runs out the row is processed as it is, the
-// status word is set, and every thread still reaches every barrier.
-// DBG adds the optional fp32 output of the reordered LayerNorm values (off the fast path).
-// GB32: gains and biases are kept as fp32 in shared memory (when they fit), else as fp16.
-enum { BAR_LN = 1, BAR_FULL0 = 2, BAR_EMPTY0 = 4 };
-constexpr long long kLnWaitBudgetCycles = 4000000000ll;
+// Bounded wait. When the budget runs out the status word is set, every later wait in the block
+// returns at once, and the caller carries on with whatever the slot holds: the loops have fixed
+// trip counts, so the kernel still ends.
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status)
+{
+    if (mbar_try_wait(bar, parity)) return;
+    const long long t0 = clock64();
+#pragma unroll 1
+    while (true) {
+#pragma unroll 1
+        for (int i = 0; i < 256; ++i)
+            if (mbar_try_wait(bar, parity)) return;
+        if (*abort_flag) return;
+        if (clock64() - t0 > kLnWaitBudgetCycles) {
+            *abort_flag = 1;
+            if (status) atomicExch(status, RPTQ_ERR_DEVICE_TIMEOUT);
+            return;
+        }
+    }
+}
+
+__device__ __forceinline__ int min_relu(int a, int b)      // max(min(a, b), 0) in one instruction
+{
+    int d;
+    asm("min.relu.s32 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
 
 struct LnParams {
     const __half* x; int64_t ldx; const __half* gamma; const __half* beta; float eps;
-    int M, C, n_units, TL, depth;
-    const uint16_t* src_tab; const UnitInfo* unit_tab;
+    int M, C, n_units, n_stats_warps, depth;
+    const uint16_t* ch_tab;      // [K_pad] channel of each padded position, C at pad positions
+    const int32_t* jidx_tab;     // [K_pad] reordered index of each padded position, -1 at pads (debug output)
+    const UnitInfo* unit_tab;
     uint8_t* codes; int64_t row_bytes; float* y_dbg; int* status;
 };
 
-// MAXT bounds the block size (512: up to 128 registers per thread; 1024: 64).
-template <int NCH, int BITS, bool DBG, int MAXT, bool GB32>
-__global__ void __launch_bounds__(MAXT)
+// Warp roles:
+//   warp 0                 lane 0 keeps the ring full: one contiguous cp.async.bulk per row (at 18-24 KB
+//                          a row, a few rows in flight per SM would leave HBM idle most of the time)
+//   warps 1 .. S           statistics: a warp takes every S-th row, reads it twice from shared memory
+//                          (mean, then the sum of squared deviations) and publishes (rstd, -mean * rstd)
+//   the other warps        gather: each thread owns one output unit. Its 32 source offsets, gains and
+//                          biases stay in registers across rows; per row it reads its 32 raw fp16
+//                          values, forms y = ((x * rstd - mean * rstd) * gain + bias) in fp32,
+//                          quantises and stores 12/16/32 contiguous bytes
+// Per ring slot three mbarriers hand the row over: landed (copy engine) -> ready (statistics) ->
+// free (all gather warps), which lets the producer refill it.
+// DBG adds the optional fp32 output of the reordered LayerNorm values (off the fast path).
+template <int BITS, bool DBG>
+__global__ void __launch_bounds__(512)
 ln_reorder_quant_kernel(const LnParams p)
 {
     extern __shared__ __align__(128) uint8_t smem_raw[];
-    const int T = blockDim.x, TL = p.TL, TG = T - TL, C = p.C;
-    const int tid = threadIdx.x;
-    const int n_chunks = C >> 3;
-    const int ybuf_stride = (C + 4 + 3) & ~3;           // C floats in split-half order + the pad slot
-    float* ybuf0 = reinterpret_cast<float*>(smem_raw);
-    uint8_t* gb = smem_raw + 2 * ybuf_stride * 4;        // gains, then biases (fp32 or fp16)
-    uint8_t* ring = gb + (GB32 ? 8 : 4) * C;             // `depth` raw rows of 2 C bytes
-    float* red = reinterpret_cast<float*>(ring + (size_t)p.depth * 2 * C);   // [2][2][32]
-    uint64_t* bars = reinterpret_cast<uint64_t*>(red + 128);                 // [depth] row landed
+    const int T = blockDim.x, C = p.C, D = p.depth, S = p.n_stats_warps;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t row_bytes_in = 2u * (uint32_t)C;
+    const uint32_t pitch = row_bytes_in + 16u;            // the half after the row is the pad source
+    uint8_t* ring = smem_raw;
+    float2* stats = reinterpret_cast<float2*>(ring + (size_t)D * pitch);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(stats + D);                  // landed[D], ready[D], free[D]
+    volatile int* s_abort = reinterpret_cast<volatile int*>(bars + 3 * D);
     const uint32_t ring_s = (uint32_t)__cvta_generic_to_shared(ring);
     const uint32_t bar_s = (uint32_t)__cvta_generic_to_shared(bars);
+    const int TG = T - 32 * (1 + S), n_gather_warps = TG >> 5;
     const int n_rows = (p.M - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;   // rows of this block
 
     if (tid == 0) {
-        // pad positions read this slot: -inf quantises to code 0 whatever the parameters
-        ybuf0[C] = -INFINITY; ybuf0[ybuf_stride + C] = -INFINITY;
-        for (int d = 0; d < p.depth; ++d) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_s + 8 * d) : "memory");
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    for (int ch = tid; ch < n_chunks; ch += T) {
-        const uint4 gv = __ldg(reinterpret_cast<const uint4*>(p.gamma + ch * 8));
-        const uint4 bv = __ldg(reinterpret_cast<const uint4*>(p.beta + ch * 8));
-        if constexpr (GB32) {
-            // four regions of one float4 per chunk (gains 0-3, gains 4-7, biases 0-3, biases 4-7) so
-            // that the LayerNorm warps' vector reads are contiguous across lanes
-            float* g = reinterpret_cast<float*>(gb);
-            const __half2* gh = reinterpret_cast<const __half2*>(&gv);
-            const __half2* bh = reinterpret_cast<const __half2*>(&bv);
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                *reinterpret_cast<float2*>(g + ((e >> 1) * n_chunks + ch) * 4 + 2 * (e & 1)) = __half22float2(gh[e]);
-                *reinterpret_cast<float2*>(g + ((2 + (e >> 1)) * n_chunks + ch) * 4 + 2 * (e & 1)) = __half22float2(bh[e]);
-            }
-        } else {
-            reinterpret_cast<uint4*>(gb)[ch] = gv;
-            reinterpret_cast<uint4*>(gb)[n_chunks + ch] = bv;
+        for (int d = 0; d < D; ++d) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_s + 8 * d) : "memory");
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_s + 8 * (D + d)) : "memory");
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar_s + 8 * (2 * D + d)), "r"(n_gather_warps) : "memory");
+            // pad positions read this half: -inf quantises to code 0 whatever the parameters
+            *reinterpret_cast<unsigned short*>(ring + (size_t)d * pitch + row_bytes_in) = 0xFC00u;
         }
+        *s_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
 
-    if (tid < TL) {
-        // ------------------------------------------------------------ LayerNorm warps
-        const int lane = tid & 31, warp = tid >> 5, nwarps = TL >> 5;
+    if (warp == 0) {
+        // ------------------------------------------------------------ producer
+        if (lane == 0) {
+            const int64_t row_step = (int64_t)gridDim.x * p.ldx;
+            const __half* src = p.x + (int64_t)blockIdx.x * p.ldx;
+            int d = 0;
+            uint32_t par = 1;                // parity to wait for on free[d]: passes at once the first time round
+            for (int k = 0; k < n_rows; ++k) {
+                mbar_wait(bar_s + 8 * (2 * D + d), par, s_abort, p.status);
+                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_s + 8 * d), "r"(row_bytes_in) : "memory");
+                asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                             ::"r"(ring_s + d * pitch), "l"(src), "r"(row_bytes_in), "r"(bar_s + 8 * d) : "memory");
+                src += row_step;
+                if (++d == D) { d = 0; par ^= 1u; }
+            }
+            // every copy has landed before the block's shared memory goes away: the statistics warps
+            // wait for each of them
+        }
+    } else if (warp <= S) {
+        // ------------------------------------------------------------ statistics warps
+        const int n_chunks = C >> 3;
         const float inv_C = 1.0f / (float)C;
-        const uint32_t row_bytes_in = 2u * (uint32_t)C;
-        // One thread keeps the ring full. Slots, parities and source pointers advance by increments:
-        // this is a single thread of dependent instructions on every row's critical path.
-        const int64_t row_step = (int64_t)gridDim.x * p.ldx;
-        const __half* next_src = p.x + (int64_t)blockIdx.x * p.ldx;
-        int next_row = 0, next_slot = 0;
-        auto issue_row = [&]() {             // row `next_row` of this block into ring slot `next_slot`
-            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_s + 8 * next_slot), "r"(row_bytes_in) : "memory");
-            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                         ::"r"(ring_s + next_slot * row_bytes_in), "l"(next_src), "r"(row_bytes_in), "r"(bar_s + 8 * next_slot) : "memory");
-            next_src += row_step;
-            ++next_row;
-            if (++next_slot == p.depth) next_slot = 0;
-        };
-        if (tid == 0)
-            while (next_row < p.depth - 1 && next_row < n_rows) issue_row();
-        int slot = 0;
-        uint32_t parity = 0;
-        for (int i = 0; i < n_rows; ++i) {
-            const int b = i & 1;
-            // Refill the slot of row i-1: every LayerNorm thread read it before that row's first barrier.
-            if (tid == 0 && next_row < n_rows) issue_row();
-            if (!mbar_try_wait(bar_s + 8 * slot, parity)) {
-                const long long t0 = clock64();
-                while (!mbar_try_wait(bar_s + 8 * slot, parity)) {
-                    if (clock64() - t0 > kLnWaitBudgetCycles) { if (p.status) atomicExch(p.status, RPTQ_ERR_DEVICE_TIMEOUT); break; }
-                }
-            }
-            const uint32_t row_s = ring_s + slot * row_bytes_in;
-            if (++slot == p.depth) { slot = 0; parity ^= 1u; }
-            float2 xf[NCH][4];
-#pragma unroll
-            for (int k = 0; k < NCH; ++k) {
-                const int ch = tid + k * TL;
-                const uint4 raw = ch < n_chunks ? lds_v4(row_s + ch * 16) : make_uint4(0, 0, 0, 0);
+        for (int k = warp - 1; k < n_rows; k += S) {
+            const int d = k % D;
+            mbar_wait(bar_s + 8 * d, (uint32_t)(k / D) & 1u, s_abort, p.status);
+            const uint4* row = reinterpret_cast<const uint4*>(ring + (size_t)d * pitch);
+            float2 s2 = make_float2(0.f, 0.f), s2b = make_float2(0.f, 0.f);
+#pragma unroll 4
+            for (int ch = lane; ch < n_chunks; ch += 32) {
+                const uint4 raw = row[ch];
                 const __half2* h = reinterpret_cast<const __half2*>(&raw);
-#pragma unroll
-                for (int e = 0; e < 4; ++e) xf[k][e] = __half22float2(h[e]);
+                s2 = add2(s2, add2(__half22float2(h[0]), __half22float2(h[1])));
+                s2b = add2(s2b, add2(__half22float2(h[2]), __half22float2(h[3])));
             }
-            float* redm = red + b * 64;
-            // mean
-            float2 s2 = make_float2(0.f, 0.f);
-#pragma unroll
-            for (int k = 0; k < NCH; ++k)
-#pragma unroll
-                for (int e = 0; e < 4; ++e) s2 = add2(s2, xf[k][e]);
-            const float s = warp_sum(s2.x + s2.y);
-            if (lane == 0) redm[warp] = s;
-            bar_sync(BAR_LN, TL);
-            float tot = 0.f;
-            for (int w = 0; w < nwarps; ++w) tot += redm[w];
-            const float mu = tot * inv_C;
-            // variance, two-pass on the registers
+            const float mu = warp_sum((s2.x + s2.y) + (s2b.x + s2b.y)) * inv_C;
             const float2 neg_mu = make_float2(-mu, -mu);
-            float2 q2 = make_float2(0.f, 0.f);
-#pragma unroll
-            for (int k = 0; k < NCH; ++k) {
-                const bool live = (tid + k * TL) < n_chunks;
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    xf[k][e] = live ? add2(xf[k][e], neg_mu) : make_float2(0.f, 0.f);
-                    q2 = fma2(xf[k][e], xf[k][e], q2);
-                }
+            float2 q2 = make_float2(0.f, 0.f), q2b = make_float2(0.f, 0.f);
+#pragma unroll 4
+            for (int ch = lane; ch < n_chunks; ch += 32) {
+                const uint4 raw = row[ch];
+                const __half2* h = reinterpret_cast<const __half2*>(&raw);
+                const float2 a = add2(__half22float2(h[0]), neg_mu), b = add2(__half22float2(h[1]), neg_mu);
+                const float2 c = add2(__half22float2(h[2]), neg_mu), e = add2(__half22float2(h[3]), neg_mu);
+                q2 = fma2(a, a, q2); q2b = fma2(b, b, q2b);
+                q2 = fma2(c, c, q2); q2b = fma2(e, e, q2b);
             }
-            const float sq = warp_sum(q2.x + q2.y);
-            if (lane == 0) redm[32 + warp] = sq;
-            bar_sync(BAR_LN, TL);
-            float tq = 0.f;
-            for (int w = 0; w < nwarps; ++w) tq += redm[32 + w];
-            const float rstd = 1.0f / sqrtf(tq * inv_C + p.eps);
-            const float2 rstd2 = make_float2(rstd, rstd);
-            // the gather of row i-2 must have finished with this buffer
-            if (i >= 2) bar_sync(BAR_EMPTY0 + b, T);
-            float* ybuf = ybuf0 + b * ybuf_stride;
-#pragma unroll
-            for (int k = 0; k < NCH; ++k) {
-                const int ch = tid + k * TL;
-                if (ch < n_chunks) {
-                    float2 g[4], bt[4];
-                    if constexpr (GB32) {
-                        const float4* g4 = reinterpret_cast<const float4*>(gb) + ch;
-                        const float4 ga = g4[0], gc = g4[n_chunks], ba = g4[2 * n_chunks], bc = g4[3 * n_chunks];
-                        g[0] = make_float2(ga.x, ga.y); g[1] = make_float2(ga.z, ga.w); g[2] = make_float2(gc.x, gc.y); g[3] = make_float2(gc.z, gc.w);
-                        bt[0] = make_float2(ba.x, ba.y); bt[1] = make_float2(ba.z, ba.w); bt[2] = make_float2(bc.x, bc.y); bt[3] = make_float2(bc.z, bc.w);
-                    } else {
-                        const uint4 gv = reinterpret_cast<const uint4*>(gb)[ch], bv = reinterpret_cast<const uint4*>(gb)[n_chunks + ch];
-                        const __half2* gh = reinterpret_cast<const __half2*>(&gv);
-                        const __half2* bh = reinterpret_cast<const __half2*>(&bv);
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) { g[e] = __half22float2(gh[e]); bt[e] = __half22float2(bh[e]); }
-                    }
-                    float2 y[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) y[e] = fma2(mul2(xf[k][e], rstd2), g[e], bt[e]);
-                    *reinterpret_cast<float4*>(ybuf + ch * 4) = make_float4(y[0].x, y[0].y, y[1].x, y[1].y);
-                    *reinterpret_cast<float4*>(ybuf + (C >> 1) + ch * 4) = make_float4(y[2].x, y[2].y, y[3].x, y[3].y);
-                }
+            const float var = warp_sum((q2.x + q2.y) + (q2b.x + q2b.y)) * inv_C;
+            const float rstd = 1.0f / sqrtf(var + p.eps);
+            if (lane == 0) {
+                stats[d] = make_float2(rstd, -mu * rstd);
+                mbar_arrive(bar_s + 8 * (D + d));            // release: the statistics are visible to whoever sees the phase
             }
-            __threadfence_block();
-            bar_arrive(BAR_FULL0 + b, T);
         }
     } else {
         // ------------------------------------------------------------ gather warps
-        const int gt = tid - TL;
-        const uint32_t ybuf_s = (uint32_t)__cvta_generic_to_shared(ybuf0);
-        const bool one_unit = p.n_units <= TG;             // the fast case: my unit's table stays in registers
-        uint32_t src_addr[32];
+        const int gt = tid - 32 * (1 + S);
+        const bool one_unit = p.n_units <= TG;             // the fast case: my unit's tables stay in registers
+        uint32_t off[32];                                  // byte offset of each source channel in a ring slot
+        float2 g2[16], b2[16];                             // gains and biases of source channels 2 i, 2 i + 1
         UnitInfo ui = {1.0f, 0, 0, 0};
+        uint32_t keep[BITS];                               // packed words with all bits set at the unit's real positions
+        const int qmax = (1 << BITS) - 1;
         auto load_unit = [&](int u) {
-            const uint4* sp = reinterpret_cast<const uint4*>(p.src_tab + u * 32);
+            const uint4* sp = reinterpret_cast<const uint4*>(p.ch_tab + u * 32);
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const uint4 v = __ldg(sp + i);
                 const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
-                    src_addr[8 * i + 2 * j] = ybuf_s + 4u * (w[j] & 0xFFFFu);
-                    src_addr[8 * i + 2 * j + 1] = ybuf_s + 4u * (w[j] >> 16);
+                    const uint32_t c0 = w[j] & 0xFFFFu, c1 = w[j] >> 16;
+                    off[8 * i + 2 * j] = 2u * c0;
+                    off[8 * i + 2 * j + 1] = 2u * c1;
+                    const bool r0 = c0 < (uint32_t)C, r1 = c1 < (uint32_t)C;
+                    g2[4 * i + j] = make_float2(r0 ? __half2float(__ldg(p.gamma + c0)) : 1.0f, r1 ? __half2float(__ldg(p.gamma + c1)) : 1.0f);
+                    b2[4 * i + j] = make_float2(r0 ? __half2float(__ldg(p.beta + c0)) : 0.0f, r1 ? __half2float(__ldg(p.beta + c1)) : 0.0f);
                 }
             }
             const uint4 t4 = __ldg(reinterpret_cast<const uint4*>(p.unit_tab + u));
             ui.inv_s = __uint_as_float(t4.x); ui.zc = (int)t4.y; ui.j0 = (int)t4.z; ui.nvalid = (int)t4.w;
+            // pad positions give code 0 even when the row's statistics are not finite
+            uint32_t full[32];
+#pragma unroll
+            for (int e = 0; e < 32; ++e) full[e] = e < ui.nvalid ? (uint32_t)qmax : 0u;
+            pack32<BITS>(full, keep);
         };
         if (one_unit && gt < p.n_units) load_unit(gt);
-        const int qmax = (1 << BITS) - 1;
+        const float2 magic2 = make_float2(12582912.0f, 12582912.0f);
         int m = blockIdx.x;
-        for (int i = 0; i < n_rows; ++i, m += gridDim.x) {
-            const int b = i & 1;
-            const uint32_t boff = (uint32_t)(b * ybuf_stride) * 4u;
-            bar_sync(BAR_FULL0 + b, T);
+        int d = 0;
+        uint32_t par = 0;
+        for (int k = 0; k < n_rows; ++k, m += gridDim.x) {
+            mbar_wait(bar_s + 8 * (D + d), par, s_abort, p.status);
+            const float2 st = stats[d];
+            const float2 rs2 = make_float2(st.x, st.x), nm2 = make_float2(st.y, st.y);
+            const uint8_t* slot = ring + (size_t)d * pitch;
             uint8_t* out_row = p.codes + (int64_t)m * p.row_bytes;
             for (int u = gt; u < p.n_units; u += TG) {
                 if (!one_unit) load_unit(u);
+                const float2 inv_s2 = make_float2(ui.inv_s, ui.inv_s);
                 uint32_t q[32];
 #pragma unroll
-                for (int e = 0; e < 32; ++e) {
-                    const float yv = lds_f32(src_addr[e] + boff);
-                    q[e] = quant_code(yv, ui.inv_s, ui.zc, qmax);
+                for (int i = 0; i < 16; ++i) {
+                    const __half h0 = *reinterpret_cast<const __half*>(slot + off[2 * i]);
+                    const __half h1 = *reinterpret_cast<const __half*>(slot + off[2 * i + 1]);
+                    const float2 xh = fma2(make_float2(__half2float(h0), __half2float(h1)), rs2, nm2);
+                    const float2 y = fma2(xh, g2[i], b2[i]);
+                    // the quantiser decision of quant_code (pack.cuh), two values at a time
+                    const float2 t = fma2(y, inv_s2, magic2);
+                    q[2 * i] = (uint32_t)min_relu(__float_as_int(t.x) + ui.zc, qmax);
+                    q[2 * i + 1] = (uint32_t)min_relu(__float_as_int(t.y) + ui.zc, qmax);
                     if constexpr (DBG) {
-                        if (e < ui.nvalid) p.y_dbg[(int64_t)m * C + ui.j0 + e] = yv;
+                        const int j0 = __ldg(p.jidx_tab + u * 32 + 2 * i), j1 = __ldg(p.jidx_tab + u * 32 + 2 * i + 1);
+                        if (j0 >= 0) p.y_dbg[(int64_t)m * C + j0] = y.x;
+                        if (j1 >= 0) p.y_dbg[(int64_t)m * C + j1] = y.y;
                     }
                 }
                 uint32_t w[BITS];
                 pack32<BITS>(q, w);
+#pragma unroll
+                for (int i = 0; i < BITS; ++i) w[i] &= keep[i];
                 if constexpr (BITS == 8) {
                     uint4* dst = reinterpret_cast<uint4*>(out_row + u * 32);
                     dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
@@ -307,35 +280,19 @@ ln_reorder_quant_kernel(const LnParams p)
                     dst[0] = w[0]; dst[1] = w[1]; dst[2] = w[2];
                 }
             }
-            if (i + 2 < n_rows) bar_arrive(BAR_EMPTY0 + b, T);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_s + 8 * (2 * D + d));     // this warp has read everything it needs from the slot
+            if (++d == D) { d = 0; par ^= 1u; }
         }
     }
 }
 
 using KernelFn = void (*)(const LnParams);
 
-template <int BITS, bool DBG, int MAXT, bool GB32>
-static KernelFn pick_kernel(int nch)
-{
-    switch (nch) {
-        case 1: return ln_reorder_quant_kernel<1, BITS, DBG, MAXT, GB32>;
-        case 2: return ln_reorder_quant_kernel<2, BITS, DBG, MAXT, GB32>;
-        case 3: return ln_reorder_quant_kernel<3, BITS, DBG, MAXT, GB32>;
-        case 4: return ln_reorder_quant_kernel<4, BITS, DBG, MAXT, GB32>;
-        case 5: case 6: return ln_reorder_quant_kernel<6, BITS, DBG, MAXT, GB32>;
-        default: return ln_reorder_quant_kernel<8, BITS, DBG, MAXT, GB32>;
-    }
-}
-template <bool DBG, int MAXT, bool GB32>
-static KernelFn pick_kernel_bits(int bits, int nch)
-{
-    return bits == 3 ? pick_kernel<3, DBG, MAXT, GB32>(nch) : bits == 4 ? pick_kernel<4, DBG, MAXT, GB32>(nch) : pick_kernel<8, DBG, MAXT, GB32>(nch);
-}
 template <bool DBG>
-static KernelFn pick_kernel_all(int bits, int nch, bool big, bool gb32)
+static KernelFn pick_kernel(int bits)
 {
-    if (big) return gb32 ? pick_kernel_bits<DBG, 1024, true>(bits, nch) : pick_kernel_bits<DBG, 1024, false>(bits, nch);
-    return gb32 ? pick_kernel_bits<DBG, 512, true>(bits, nch) : pick_kernel_bits<DBG, 512, false>(bits, nch);
+    return bits == 3 ? ln_reorder_quant_kernel<3, DBG> : bits == 4 ? ln_reorder_quant_kernel<4, DBG> : ln_reorder_quant_kernel<8, DBG>;
 }
 
 // Launch shape of one kernel instance on one device, computed on first use (the attribute and
@@ -374,43 +331,34 @@ extern "C" int rptq_ln_reorder_quant(const rptq_layout_t* L, const void* x, int6
     if (L->device < 0 || cudaGetDevice(&dev) != cudaSuccess) return RPTQ_ERR_CUDA;
     if (dev != L->device) return RPTQ_ERR_INVALID_ARG;
 
-    // Shared memory: two normalised rows (8 C bytes), gains and biases (8 C as fp32, else 4 C as
-    // fp16), and a ring of raw rows (2 C each), at least 2 and at most 6 deep.
+    // Shared memory: a ring of raw rows (2 C bytes and the pad source each), as deep as fits up to
+    // 16 rows, with two floats and three barriers per slot.
     const int C = L->C;
-    const size_t fixed = (size_t)2 * ((C + 4 + 3) & ~3) * 4 + 512 + 64;
+    const size_t pitch = (size_t)2 * C + 16;
     const size_t limit = 227 * 1024;
-    bool gb32 = fixed + (size_t)8 * C + (size_t)4 * 2 * C <= limit;
-    const size_t gb_bytes = (size_t)(gb32 ? 8 : 4) * C;
-    if (fixed + gb_bytes + (size_t)2 * 2 * C > limit) return RPTQ_ERR_UNSUPPORTED;
-    int depth = (int)((limit - fixed - gb_bytes) / ((size_t)2 * C));
-    depth = depth > 6 ? 6 : depth;
-    const size_t smem = fixed + gb_bytes + (size_t)depth * 2 * C;
+    int depth = (int)((limit - 64) / (pitch + 32));
+    if (depth < 2) return RPTQ_ERR_UNSUPPORTED;
+    depth = depth > 16 ? 16 : depth;
+    const size_t smem = (size_t)depth * (pitch + 32) + 64;
 
-    // Gather threads: one per output unit up to 512 (beyond that each thread loops over units).
-    // LayerNorm threads: a thread holds NCH chunks of 8 channels in registers. Blocks of up to 512
-    // threads may use 128 registers per thread (NCH <= 6); larger blocks only 64 (NCH <= 3 wanted).
-    const int n_chunks = C / 8;
-    const int TG = L->n_units >= 512 ? 512 : (L->n_units + 31) / 32 * 32;
-    int TL = 64;
-    while (TL + TG + 32 <= 512 && (n_chunks + TL - 1) / TL > 3) TL += 32;
-    const bool big = (n_chunks + TL - 1) / TL > 6;
-    if (big) {
-        TL = 64;
-        while (TL + TG + 32 <= 1024 && (n_chunks + TL - 1) / TL > 3) TL += 32;
-    }
-    const int nch = (n_chunks + TL - 1) / TL;
-    if (nch > 8) return RPTQ_ERR_UNSUPPORTED;
-    const int T = TL + TG;
+    // One gather thread per output unit where that fits beside four statistics warps in a block
+    // of 512 threads (128 registers each); wider layouts get two statistics warps, and beyond 416
+    // units each gather thread loops over several units and reloads its tables.
+    const int want = (L->n_units + 31) / 32 * 32;
+    int TG, S;
+    if (want <= 352) { TG = want; S = 4; }
+    else { TG = want <= 416 ? want : 416; S = 2; }
+    const int T = 32 * (1 + S) + TG;
 
-    KernelFn fn = y_dbg ? pick_kernel_all<true>(L->bits, nch, big, gb32) : pick_kernel_all<false>(L->bits, nch, big, gb32);
+    KernelFn fn = y_dbg ? pick_kernel<true>(L->bits) : pick_kernel<false>(L->bits);
     int blocks = 0;
     const int rc = planned_blocks(reinterpret_cast<const void*>(fn), dev, T, smem, &blocks);
     if (rc != RPTQ_OK) return rc;
     LnParams p{};
     p.x = static_cast<const __half*>(x); p.ldx = ldx; p.gamma = static_cast<const __half*>(gamma);
-    p.beta = static_cast<const __half*>(beta); p.eps = eps; p.M = M; p.C = C; p.n_units = L->n_units; p.TL = TL;
-    p.depth = depth; p.src_tab = L->d_src; p.unit_tab = L->d_unit; p.codes = static_cast<uint8_t*>(codes);
-    p.row_bytes = L->row_bytes; p.y_dbg = y_dbg; p.status = device_status_word();
+    p.beta = static_cast<const __half*>(beta); p.eps = eps; p.M = M; p.C = C; p.n_units = L->n_units;
+    p.n_stats_warps = S; p.depth = depth; p.ch_tab = L->d_src; p.jidx_tab = L->d_jidx; p.unit_tab = L->d_unit;
+    p.codes = static_cast<uint8_t*>(codes); p.row_bytes = L->row_bytes; p.y_dbg = y_dbg; p.status = device_status_word();
     fn<<<M < blocks ? M : blocks, T, smem, static_cast<cudaStream_t>(stream)>>>(p);
     return cudaGetLastError() == cudaSuccess ? RPTQ_OK : RPTQ_ERR_CUDA;
 }

@@ -26,11 +26,6 @@ enum : uint8_t { STEP_FIRST = 1, STEP_LAST = 2, STEP_SKIP = 4, STEP_BUF = 8 };
 
 constexpr int kMaxGemmSegments = 1024;
 
-// Shared-memory slot (in floats) of channel c of a normalised row in rptq_ln_reorder_quant. The
-// two 16-byte halves of each 8-channel chunk live in separate regions so that both vector stores
-// of a warp are contiguous across lanes; slot C holds the value that pad positions read.
-__host__ __device__ inline int ybuf_addr(int c, int C) { return ((c >> 3) << 2) + (c & 3) + ((c >> 2) & 1) * (C >> 1); }
-
 // Byte offset of the 64-byte piece (row n, K block kb) in the tile-major packed weight buffer.
 __host__ __device__ inline int64_t weight_tile_offset(int64_t n, int kb, int n_kb) { return ((n >> 7) * n_kb + kb) * 8192 + (n & 127) * 64; }
 
@@ -46,7 +41,8 @@ struct rptq_layout {
     std::vector<int32_t> unit_cluster;   // [n_units] owning cluster, -1 past the last cluster
     std::vector<float> scale;
     // device tables
-    uint16_t* d_src = nullptr;          // [K_pad] ybuf_addr of each padded position's channel, C = pad
+    uint16_t* d_src = nullptr;          // [K_pad] channel at each padded position, C at pads
+    int32_t* d_jidx = nullptr;          // [K_pad] reordered index at each padded position, -1 at pads
     rptq::UnitInfo* d_unit = nullptr;   // [n_units]
     uint8_t* d_step_flags = nullptr;    // [n_units]
     float* d_seg_scale = nullptr;       // [n_seg]  s_c of the non-empty clusters, in the order their last steps come

@@ -46,7 +46,11 @@ def test_layout_validation_and_padded_offsets(binding):
     for c in range(g):
         want_uc[off[c] // 32:off[c + 1] // 32] = c
     assert np.array_equal(L.unit_cluster, want_uc)
-    assert np.array_equal(L.contiguous_position(), np.arange(k_pad))
+    # within a cluster the library places the channels as it likes; contiguous_position() maps back
+    m = L.contiguous_position()
+    assert sorted(m.tolist()) == list(range(k_pad))
+    for c in range(g):
+        assert np.all((m[off[c]:off[c + 1]] >= off[c]) & (m[off[c]:off[c + 1]] < off[c + 1]))
     off2, k_pad2 = calibration.segment_offsets(size)
     assert k_pad2 == k_pad and np.array_equal(off2, off)
     bad = perm.copy(); bad[3] = bad[4]
@@ -94,19 +98,28 @@ def test_weight_pack_matches_the_oracle_bit_for_bit(binding):
     for op in (None, out_perm):
         packed, s_w, wsum = binding.weight_pack(L, W, op, n_pad)
         w_codes, s_w_o, wsum_o = oracle.weight_quantize(W, perm, size, op, n_pad)
-        assert np.array_equal(packed, oracle.pack_weights(w_codes))
+        assert np.array_equal(packed, oracle.pack_weights(np.ascontiguousarray(w_codes[:, L.contiguous_position()])))
         assert np.array_equal(s_w, s_w_o) and np.array_equal(wsum, wsum_o)
     with pytest.raises(binding.RptqError):
         binding.weight_pack(L, W, np.zeros(n_pad, np.int32), n_pad)
-    # the padded index of a layout is what places a previous layer's rows for re-quantisation
+    # the padded index of a layout is what places a previous layer's rows for re-quantisation:
+    # every channel appears once, inside its own cluster's positions, pads only at a cluster's end
     idx = L.padded_index()
     off, _ = oracle.segment_offsets(size)
+    assert sorted(idx[idx >= 0].tolist()) == list(range(C))
+    j = 0
+    for c in range(g):
+        seg = idx[off[c]:off[c + 1]]
+        assert sorted(seg[:size[c]].tolist()) == sorted(perm[j:j + size[c]].tolist()) and np.all(seg[size[c]:] == -1)
+        j += size[c]
+    assert np.all(idx[off[g]:] == -1)
+    # the same array in the oracle's order, moved by contiguous_position(), is the oracle's padded index
     want = np.full(L.K_pad, -1, np.int32)
     j = 0
     for c in range(g):
         want[off[c]:off[c] + size[c]] = perm[j:j + size[c]]
         j += size[c]
-    assert np.array_equal(idx, want)
+    assert np.array_equal(idx, want[L.contiguous_position()])
 
 
 def test_interleaved_unit_order(binding):
@@ -146,10 +159,14 @@ def test_interleaved_unit_order(binding):
     # larger clusters keep their relative order and the order of their own units
     firsts = [int(np.argmax(uc == c)) for c in range(g) if units[c] > 2]
     assert firsts == sorted(firsts)
-    # every channel sits in a unit of its cluster, in the order of S
-    idx_c, idx_i, m = Lc.padded_index(), Li.padded_index(), Li.contiguous_position()
-    assert np.array_equal(idx_i, idx_c[m])
+    # every channel sits once, in a unit of its own cluster
+    idx_i, m = Li.padded_index(), Li.contiguous_position()
     assert sorted(idx_i[idx_i >= 0].tolist()) == list(range(C))
+    cluster_of = np.empty(C, np.int64)
+    cluster_of[perm] = np.repeat(np.arange(g), size)
+    real = idx_i >= 0
+    assert np.array_equal(np.repeat(uc, 32)[real], cluster_of[idx_i[real]])
+    assert sorted(m.tolist()) == list(range(Li.K_pad))
     # packed weights: the oracle's codes with their columns moved to this order
     W = rng.normal(size=(70, C)).astype(np.float32)
     packed, s_w, wsum = binding.weight_pack(Li, W, None, 72)
@@ -159,7 +176,7 @@ def test_interleaved_unit_order(binding):
     # fewer than two small clusters: nothing to interleave
     size2 = np.array([100, 60, 96], np.int32)
     L2 = binding.Layout(rng.permutation(256).astype(np.int32), size2, scale[:3], zero[:3], 4, order=binding.ORDER_INTERLEAVED)
-    assert np.array_equal(L2.contiguous_position(), np.arange(L2.K_pad))
+    assert np.array_equal(L2.unit_cluster, binding.Layout(L2._perm, size2, scale[:3], zero[:3], 4).unit_cluster)
     with pytest.raises(binding.RptqError):
         binding.Layout(perm, size, scale, zero, bits, order=2)
 

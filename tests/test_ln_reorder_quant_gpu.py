@@ -36,12 +36,12 @@ def _run(layout, x16, gamma16, beta16, want_y=True, ldx=None, stream=None):
     return codes_h[:M], y_h
 
 
-def _check_against_oracle(x16, gamma16, beta16, perm, size, scale32, zero, bits, packed, y_dbg, full_rate=0.9999, pos=None):
+def _check_against_oracle(x16, gamma16, beta16, perm, size, scale32, zero, bits, packed, y_dbg, full_rate=0.9999, pos=None, L=None):
     """`pos`: the layout's contiguous_position() when its unit order is not the contiguous one (the
     oracle's codes are in contiguous order)."""
     M, C = x16.shape
     _, k_pad = oracle.segment_offsets(size)
-    pos = np.arange(k_pad) if pos is None else pos
+    pos = L.contiguous_position() if pos is None else pos
     got = oracle.unpack(packed, k_pad, bits)[:, np.argsort(pos)]          # back to contiguous order
     # (1) the decision, bit for bit, from the kernel's own fp32 LayerNorm outputs
     want32 = oracle.quantize_f32(y_dbg, size, scale32, zero, bits)
@@ -90,7 +90,7 @@ def test_small_and_ragged_shapes_all_bit_widths(bits, M):
     gm = rng.lognormal(0, 0.5, C).astype(np.float16)
     bt = rng.normal(size=C).astype(np.float16)
     packed, y_dbg = _run(L, x, gm, bt, ldx=C + 24)
-    _check_against_oracle(x, gm, bt, perm, size, scale, zero, bits, packed, y_dbg, full_rate=0.999)
+    _check_against_oracle(x, gm, bt, perm, size, scale, zero, bits, packed, y_dbg, full_rate=0.999, L=L)
 
 
 @pytest.mark.parametrize("bits", [3, 4, 8])
@@ -114,7 +114,7 @@ def test_degenerate_clusterings(bits):
     for perm_, size_, scale_, zero_ in (one, per_ch, empty):
         L = binding.Layout(perm_, size_, scale_, zero_, bits)
         packed, y_dbg = _run(L, x, gm, bt)
-        _check_against_oracle(x, gm, bt, perm_, size_, scale_, zero_, bits, packed, y_dbg, full_rate=0.999)
+        _check_against_oracle(x, gm, bt, perm_, size_, scale_, zero_, bits, packed, y_dbg, full_rate=0.999, L=L)
 
 
 def test_wide_rows_take_the_multi_unit_path_and_zero_tokens_launch_nothing():
@@ -129,7 +129,7 @@ def test_wide_rows_take_the_multi_unit_path_and_zero_tokens_launch_nothing():
     gm = rng.lognormal(0, 0.5, C).astype(np.float16)
     bt = rng.normal(size=C).astype(np.float16)
     packed, y_dbg = _run(L, x, gm, bt)
-    _check_against_oracle(x, gm, bt, perm, size, scale, zero, bits, packed, y_dbg, full_rate=0.999)
+    _check_against_oracle(x, gm, bt, perm, size, scale, zero, bits, packed, y_dbg, full_rate=0.999, L=L)
     codes = torch.full((4, L.row_bytes), CANARY, dtype=torch.uint8, device="cuda")
     xd = torch.zeros((1, C), dtype=torch.float16, device="cuda")
     binding.ln_reorder_quant(L, xd, torch.from_numpy(gm).cuda(), torch.from_numpy(bt).cuda(), EPS, codes, None, M=0)
@@ -150,8 +150,5 @@ def test_non_finite_inputs_still_give_in_range_codes():
     packed, _ = _run(L, x, gm, bt)
     got = oracle.unpack(packed, L.K_pad, bits)
     assert got.max() <= 15
-    off, _ = oracle.segment_offsets(size)
-    pads = np.ones(L.K_pad, bool)
-    for c in range(3):
-        pads[off[c]:off[c] + size[c]] = False
+    pads = L.padded_index() < 0
     assert not got[:, pads].any()

@@ -31,7 +31,9 @@ def _problem(rng, M, N, C, g, bits):
     a = np.zeros((M, k_pad), np.uint8)
     for c in range(g):
         a[:, off[c]:off[c] + size[c]] = rng.integers(0, 1 << bits, size=(M, size[c]))
-    dev = dict(L=L, a=torch.from_numpy(oracle.pack(a, bits)).cuda(), w=torch.from_numpy(oracle.pack_weights(w_codes)).cuda(),
+    m = L.contiguous_position()          # the oracle's column order -> the layout's
+    dev = dict(L=L, a=torch.from_numpy(oracle.pack(np.ascontiguousarray(a[:, m]), bits)).cuda(),
+               w=torch.from_numpy(oracle.pack_weights(np.ascontiguousarray(w_codes[:, m]))).cuda(),
                s_w=torch.from_numpy(s_w).cuda(), wsum=torch.from_numpy(wsum).cuda(),
                bias=torch.from_numpy((rng.normal(size=N) * 0.05).astype(np.float32)).cuda())
     want = oracle.cluster_gemm(a, w_codes, size, scale.astype(np.float64), zero, s_w, wsum, bias=dev["bias"].cpu().numpy())
