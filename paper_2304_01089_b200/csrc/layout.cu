@@ -262,6 +262,9 @@ int rptq_layout_create(rptq_layout_t** out, int C, int g, int bits, const int32_
         for (int w0 = 0; w0 < L->n_units; w0 += 32)
             for (int e = 0; e < 32; ++e) {
                 uint32_t used = 0;
+                // lanes whose unit has no element e read the pad source behind the row: keep its bank free
+                for (int l = 0; l < 32 && w0 + l < L->n_units; ++l)
+                    if (e >= unit[w0 + l].nvalid) used |= 1u << ((C >> 1) & 31);
                 for (int l = 0; l < 32 && w0 + l < L->n_units; ++l) {
                     const int u = w0 + l, c = L->unit_cluster[u];
                     if (c < 0 || e >= unit[u].nvalid) continue;

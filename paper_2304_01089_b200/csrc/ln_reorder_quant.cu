@@ -146,10 +146,25 @@ ln_reorder_quant_kernel(const LnParams p)
         *s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    // Gains and biases pass through ring slots 0 and 1 (coalesced loads) so that the gather threads
+    // can pick their own channels' values from shared memory; scattered 2-byte global loads for
+    // 64 values per thread would cost more than a few hundred rows of the kernel proper.
+    {
+        uint4* g_s = reinterpret_cast<uint4*>(ring);
+        uint4* b_s = reinterpret_cast<uint4*>(ring + pitch);
+        for (int ch = tid; ch < (C >> 3); ch += T) {
+            g_s[ch] = __ldg(reinterpret_cast<const uint4*>(p.gamma) + ch);
+            b_s[ch] = __ldg(reinterpret_cast<const uint4*>(p.beta) + ch);
+        }
+    }
     __syncthreads();
+    const __half* gamma_s = reinterpret_cast<const __half*>(ring);
+    const __half* beta_s = reinterpret_cast<const __half*>(ring + pitch);
+    const bool tables_in_regs = p.n_units <= TG;       // else the gather threads reload tables per unit, from global memory
 
     if (warp == 0) {
         // ------------------------------------------------------------ producer
+        __syncthreads();                     // the gather threads have taken their gains and biases out of the ring
         if (lane == 0) {
             const int64_t row_step = (int64_t)gridDim.x * p.ldx;
             const __half* src = p.x + (int64_t)blockIdx.x * p.ldx;
@@ -168,6 +183,7 @@ ln_reorder_quant_kernel(const LnParams p)
         }
     } else if (warp <= S) {
         // ------------------------------------------------------------ statistics warps
+        __syncthreads();
         const int n_chunks = C >> 3;
         const float inv_C = 1.0f / (float)C;
         for (int k = warp - 1; k < n_rows; k += S) {
@@ -204,13 +220,13 @@ ln_reorder_quant_kernel(const LnParams p)
     } else {
         // ------------------------------------------------------------ gather warps
         const int gt = tid - 32 * (1 + S);
-        const bool one_unit = p.n_units <= TG;             // the fast case: my unit's tables stay in registers
+        const bool one_unit = tables_in_regs;              // the fast case: my unit's tables stay in registers
         uint32_t off[32];                                  // byte offset of each source channel in a ring slot
         float2 g2[16], b2[16];                             // gains and biases of source channels 2 i, 2 i + 1
         UnitInfo ui = {1.0f, 0, 0, 0};
         uint32_t keep[BITS];                               // packed words with all bits set at the unit's real positions
         const int qmax = (1 << BITS) - 1;
-        auto load_unit = [&](int u) {
+        auto load_unit = [&](int u, const __half* gamma, const __half* beta) {
             const uint4* sp = reinterpret_cast<const uint4*>(p.ch_tab + u * 32);
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
@@ -222,8 +238,8 @@ ln_reorder_quant_kernel(const LnParams p)
                     off[8 * i + 2 * j] = 2u * c0;
                     off[8 * i + 2 * j + 1] = 2u * c1;
                     const bool r0 = c0 < (uint32_t)C, r1 = c1 < (uint32_t)C;
-                    g2[4 * i + j] = make_float2(r0 ? __half2float(__ldg(p.gamma + c0)) : 1.0f, r1 ? __half2float(__ldg(p.gamma + c1)) : 1.0f);
-                    b2[4 * i + j] = make_float2(r0 ? __half2float(__ldg(p.beta + c0)) : 0.0f, r1 ? __half2float(__ldg(p.beta + c1)) : 0.0f);
+                    g2[4 * i + j] = make_float2(r0 ? __half2float(gamma[c0]) : 1.0f, r1 ? __half2float(gamma[c1]) : 1.0f);
+                    b2[4 * i + j] = make_float2(r0 ? __half2float(beta[c0]) : 0.0f, r1 ? __half2float(beta[c1]) : 0.0f);
                 }
             }
             const uint4 t4 = __ldg(reinterpret_cast<const uint4*>(p.unit_tab + u));
@@ -234,7 +250,8 @@ ln_reorder_quant_kernel(const LnParams p)
             for (int e = 0; e < 32; ++e) full[e] = e < ui.nvalid ? (uint32_t)qmax : 0u;
             pack32<BITS>(full, keep);
         };
-        if (one_unit && gt < p.n_units) load_unit(gt);
+        if (one_unit && gt < p.n_units) load_unit(gt, gamma_s, beta_s);
+        __syncthreads();
         const float2 magic2 = make_float2(12582912.0f, 12582912.0f);
         int m = blockIdx.x;
         int d = 0;
@@ -246,7 +263,7 @@ ln_reorder_quant_kernel(const LnParams p)
             const uint8_t* slot = ring + (size_t)d * pitch;
             uint8_t* out_row = p.codes + (int64_t)m * p.row_bytes;
             for (int u = gt; u < p.n_units; u += TG) {
-                if (!one_unit) load_unit(u);
+                if (!one_unit) load_unit(u, p.gamma, p.beta);
                 const float2 inv_s2 = make_float2(ui.inv_s, ui.inv_s);
                 uint32_t q[32];
 #pragma unroll
