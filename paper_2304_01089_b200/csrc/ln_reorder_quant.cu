@@ -71,6 +71,7 @@ constexpr long long kLnWaitBudgetCycles = 4000000000ll;   // about two seconds a
 // Bounded wait. When the budget runs out the status word is set, every later wait in the block
 // returns at once, and the caller carries on with whatever the slot holds: the loops have fixed
 // trip counts, so the kernel still ends.
+template <bool BACK_OFF = false>
 __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status)
 {
     if (mbar_try_wait(bar, parity)) return;
@@ -78,8 +79,10 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatil
 #pragma unroll 1
     while (true) {
 #pragma unroll 1
-        for (int i = 0; i < 256; ++i)
+        for (int i = 0; i < 256; ++i) {
             if (mbar_try_wait(bar, parity)) return;
+            if constexpr (BACK_OFF) __nanosleep(200);    // many warps wait here: leave the issue slots to the others
+        }
         if (*abort_flag) return;
         if (clock64() - t0 > kLnWaitBudgetCycles) {
             *abort_flag = 1;
@@ -87,13 +90,6 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatil
             return;
         }
     }
-}
-
-__device__ __forceinline__ int min_relu(int a, int b)      // max(min(a, b), 0) in one instruction
-{
-    int d;
-    asm("min.relu.s32 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
-    return d;
 }
 
 struct LnParams {
@@ -257,7 +253,7 @@ ln_reorder_quant_kernel(const LnParams p)
         int d = 0;
         uint32_t par = 0;
         for (int k = 0; k < n_rows; ++k, m += gridDim.x) {
-            mbar_wait(bar_s + 8 * (D + d), par, s_abort, p.status);
+            mbar_wait<true>(bar_s + 8 * (D + d), par, s_abort, p.status);
             const float2 st = stats[d];
             const float2 rs2 = make_float2(st.x, st.x), nm2 = make_float2(st.y, st.y);
             const uint8_t* slot = ring + (size_t)d * pitch;
@@ -265,7 +261,7 @@ ln_reorder_quant_kernel(const LnParams p)
             for (int u = gt; u < p.n_units; u += TG) {
                 if (!one_unit) load_unit(u, p.gamma, p.beta);
                 const float2 inv_s2 = make_float2(ui.inv_s, ui.inv_s);
-                uint32_t q[32];
+                int q[32];                   // rne(y / s) + z, not yet clamped
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
                     const __half h0 = *reinterpret_cast<const __half*>(slot + off[2 * i]);
@@ -274,8 +270,8 @@ ln_reorder_quant_kernel(const LnParams p)
                     const float2 y = fma2(xh, g2[i], b2[i]);
                     // the quantiser decision of quant_code (pack.cuh), two values at a time
                     const float2 t = fma2(y, inv_s2, magic2);
-                    q[2 * i] = (uint32_t)min_relu(__float_as_int(t.x) + ui.zc, qmax);
-                    q[2 * i + 1] = (uint32_t)min_relu(__float_as_int(t.y) + ui.zc, qmax);
+                    q[2 * i] = __float_as_int(t.x) + ui.zc;
+                    q[2 * i + 1] = __float_as_int(t.y) + ui.zc;
                     if constexpr (DBG) {
                         const int j0 = __ldg(p.jidx_tab + u * 32 + 2 * i), j1 = __ldg(p.jidx_tab + u * 32 + 2 * i + 1);
                         if (j0 >= 0) p.y_dbg[(int64_t)m * C + j0] = y.x;
@@ -283,7 +279,7 @@ ln_reorder_quant_kernel(const LnParams p)
                     }
                 }
                 uint32_t w[BITS];
-                pack32<BITS>(q, w);
+                pack32_sat<BITS>(q, w);      // clamps to [0, 2^BITS - 1] and packs
 #pragma unroll
                 for (int i = 0; i < BITS; ++i) w[i] &= keep[i];
                 if constexpr (BITS == 8) {
@@ -363,7 +359,8 @@ extern "C" int rptq_ln_reorder_quant(const rptq_layout_t* L, const void* x, int6
     // units each gather thread loops over several units and reloads its tables.
     const int want = (L->n_units + 31) / 32 * 32;
     int TG, S;
-    if (want <= 352) { TG = want; S = 4; }
+    if (want <= 320) { TG = want; S = 5; }
+    else if (want <= 352) { TG = want; S = 4; }
     else { TG = want <= 416 ? want : 416; S = 2; }
     const int T = 32 * (1 + S) + TG;
 

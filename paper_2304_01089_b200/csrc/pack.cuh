@@ -40,4 +40,44 @@ __device__ __forceinline__ void pack32(const uint32_t (&q)[32], uint32_t (&w)[BI
     }
 }
 
+// The same words from UNCLAMPED integers: the saturating pack instruction clamps to [0, 15] (or
+// [0, 255]) and appends two codes per instruction, d = (c << 8) | (sat(a) << 4) | sat(b) for 4-bit
+// fields and d = (c << 16) | (sat(a) << 8) | sat(b) for bytes; 3-bit codes take one min first.
+__device__ __forceinline__ uint32_t sat_pack_u4(int a, int b, uint32_t c)
+{
+    uint32_t d;
+    asm("cvt.pack.sat.u4.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+__device__ __forceinline__ uint32_t sat_pack_u8(int a, int b, uint32_t c)
+{
+    uint32_t d;
+    asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+__device__ __forceinline__ uint32_t sat_nibble_word(const int* v)     // 8 integers -> one 4-bit-layout word
+{
+    uint32_t d = sat_pack_u4(v[7], v[3], 0u);
+    d = sat_pack_u4(v[6], v[2], d);
+    d = sat_pack_u4(v[5], v[1], d);
+    return sat_pack_u4(v[4], v[0], d);
+}
+template <int BITS>
+__device__ __forceinline__ void pack32_sat(int (&v)[32], uint32_t (&w)[BITS])
+{
+    if constexpr (BITS == 8) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) w[i] = sat_pack_u8(v[4 * i + 1], v[4 * i], sat_pack_u8(v[4 * i + 3], v[4 * i + 2], 0u));
+    } else if constexpr (BITS == 4) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) w[i] = sat_nibble_word(v + 8 * i);
+    } else {
+#pragma unroll
+        for (int e = 0; e < 32; ++e) v[e] = min(v[e], 7);
+        const uint32_t tail = sat_nibble_word(v + 24);
+#pragma unroll
+        for (int j = 0; j < 3; ++j) w[j] = sat_nibble_word(v + 8 * j) | (((tail >> j) & 0x11111111u) << 3);
+    }
+}
+
 }  // namespace rptq
