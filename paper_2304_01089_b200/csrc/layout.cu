@@ -201,7 +201,7 @@ int rptq_layout_create(rptq_layout_t** out, int C, int g, int bits, const int32_
         for (int c = 0; c < g; ++c) if (n_units_of[c] > 0) runs.push_back({c, 0, n_units_of[c]});
     }
 
-    std::vector<uint16_t> src((size_t)k_pad, (uint16_t)C);       // channel at each position, C at pads
+    std::vector<uint16_t> src((size_t)k_pad, 0);                 // channel read for each position (at pads: any, the code is masked)
     std::vector<int32_t> jidx((size_t)k_pad, -1);                // reordered index at each position, -1 at pads
     std::vector<UnitInfo> unit((size_t)L->n_units);
     std::vector<uint8_t> flags((size_t)L->n_units, STEP_SKIP);
@@ -262,9 +262,7 @@ int rptq_layout_create(rptq_layout_t** out, int C, int g, int bits, const int32_
         for (int w0 = 0; w0 < L->n_units; w0 += 32)
             for (int e = 0; e < 32; ++e) {
                 uint32_t used = 0;
-                // lanes whose unit has no element e read the pad source behind the row: keep its bank free
-                for (int l = 0; l < 32 && w0 + l < L->n_units; ++l)
-                    if (e >= unit[w0 + l].nvalid) used |= 1u << ((C >> 1) & 31);
+                int first_real = -1;             // channel read by the first lane that has an element e
                 for (int l = 0; l < 32 && w0 + l < L->n_units; ++l) {
                     const int u = w0 + l, c = L->unit_cluster[u];
                     if (c < 0 || e >= unit[u].nvalid) continue;
@@ -283,7 +281,12 @@ int rptq_layout_create(rptq_layout_t** out, int C, int g, int bits, const int32_
                     L->pos[j] = u * 32 + e;
                     src[u * 32 + e] = (uint16_t)perm_host[j];
                     jidx[u * 32 + e] = j;
+                    if (first_real < 0) first_real = perm_host[j];
                 }
+                // Lanes whose unit has no element e still execute the read; their codes are masked
+                // to zero afterwards, so they read what another lane reads (a broadcast costs nothing).
+                for (int l = 0; l < 32 && w0 + l < L->n_units; ++l)
+                    if (e >= unit[w0 + l].nvalid) src[(w0 + l) * 32 + e] = (uint16_t)(first_real < 0 ? 0 : first_real);
             }
     }
 

@@ -95,7 +95,7 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatil
 struct LnParams {
     const __half* x; int64_t ldx; const __half* gamma; const __half* beta; float eps;
     int M, C, n_units, n_stats_warps, depth;
-    const uint16_t* ch_tab;      // [K_pad] channel of each padded position, C at pad positions
+    const uint16_t* ch_tab;      // [K_pad] channel read for each padded position (pads: any channel, masked later)
     const int32_t* jidx_tab;     // [K_pad] reordered index of each padded position, -1 at pads (debug output)
     const UnitInfo* unit_tab;
     uint8_t* codes; int64_t row_bytes; float* y_dbg; int* status;
@@ -121,7 +121,7 @@ ln_reorder_quant_kernel(const LnParams p)
     const int T = blockDim.x, C = p.C, D = p.depth, S = p.n_stats_warps;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t row_bytes_in = 2u * (uint32_t)C;
-    const uint32_t pitch = row_bytes_in + 16u;            // the half after the row is the pad source
+    const uint32_t pitch = row_bytes_in + 16u;            // 16 spare bytes keep successive slots 4 banks apart
     uint8_t* ring = smem_raw;
     float2* stats = reinterpret_cast<float2*>(ring + (size_t)D * pitch);
     uint8_t* zero16 = ring + (size_t)D * pitch + ((8 * (size_t)D + 15) & ~(size_t)15);   // 16 zero bytes, 16-byte aligned
@@ -137,8 +137,6 @@ ln_reorder_quant_kernel(const LnParams p)
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_s + 8 * d) : "memory");
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_s + 8 * (D + d)) : "memory");
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar_s + 8 * (2 * D + d)), "r"(n_gather_warps) : "memory");
-            // pad positions read this half: -inf quantises to code 0 whatever the parameters
-            *reinterpret_cast<unsigned short*>(ring + (size_t)d * pitch + row_bytes_in) = 0xFC00u;
         }
         *s_abort = 0;
         *reinterpret_cast<uint4*>(zero16) = make_uint4(0u, 0u, 0u, 0u);
@@ -246,14 +244,13 @@ ln_reorder_quant_kernel(const LnParams p)
                     const uint32_t c0 = w[j] & 0xFFFFu, c1 = w[j] >> 16;
                     off[8 * i + 2 * j] = 2u * c0;
                     off[8 * i + 2 * j + 1] = 2u * c1;
-                    const bool r0 = c0 < (uint32_t)C, r1 = c1 < (uint32_t)C;
-                    g2[4 * i + j] = make_float2(r0 ? __half2float(gamma[c0]) : 1.0f, r1 ? __half2float(gamma[c1]) : 1.0f);
-                    b2[4 * i + j] = make_float2(r0 ? __half2float(beta[c0]) : 0.0f, r1 ? __half2float(beta[c1]) : 0.0f);
+                    g2[4 * i + j] = make_float2(__half2float(gamma[c0]), __half2float(gamma[c1]));
+                    b2[4 * i + j] = make_float2(__half2float(beta[c0]), __half2float(beta[c1]));
                 }
             }
             const uint4 t4 = __ldg(reinterpret_cast<const uint4*>(p.unit_tab + u));
             ui.inv_s = __uint_as_float(t4.x); ui.zc = (int)t4.y; ui.j0 = (int)t4.z; ui.nvalid = (int)t4.w;
-            // pad positions give code 0 even when the row's statistics are not finite
+            // pad positions read some real channel (the layout picks one that costs no bank conflict); their codes are masked to 0
             uint32_t full[32];
 #pragma unroll
             for (int e = 0; e < 32; ++e) full[e] = e < ui.nvalid ? (uint32_t)qmax : 0u;
@@ -357,7 +354,7 @@ extern "C" int rptq_ln_reorder_quant(const rptq_layout_t* L, const void* x, int6
     if (L->device < 0 || cudaGetDevice(&dev) != cudaSuccess) return RPTQ_ERR_CUDA;
     if (dev != L->device) return RPTQ_ERR_INVALID_ARG;
 
-    // Shared memory: a ring of raw rows (2 C bytes and the pad source each), as deep as fits up to
+    // Shared memory: a ring of raw rows (2 C + 16 bytes each), as deep as fits up to
     // 16 rows, with two floats and three barriers per slot.
     const int C = L->C;
     const size_t pitch = (size_t)2 * C + 16;

@@ -41,7 +41,7 @@ struct rptq_layout {
     std::vector<int32_t> unit_cluster;   // [n_units] owning cluster, -1 past the last cluster
     std::vector<float> scale;
     // device tables
-    uint16_t* d_src = nullptr;          // [K_pad] channel at each padded position, C at pads
+    uint16_t* d_src = nullptr;          // [K_pad] channel read for each padded position (at pads: some channel, the code is masked)
     int32_t* d_jidx = nullptr;          // [K_pad] reordered index at each padded position, -1 at pads
     rptq::UnitInfo* d_unit = nullptr;   // [n_units]
     uint8_t* d_step_flags = nullptr;    // [n_units]
