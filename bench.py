@@ -29,10 +29,10 @@ sys.path.insert(0, ROOT)
 WORKLOAD = "opt-66b"
 EPS = 1e-5
 # dram__bytes_read + dram__bytes_write of one FC1 GEMM launch at 4096 tokens, from the ncu capture
-# summarised in profiles/cluster_gemm_opt66b_fc1_tokens512.txt: measured at 512 tokens (191.6 MB read,
-# of which 186.4 MB are the packed weights, read once whatever the token count) with the
-# token-proportional parts (codes in, fp16 output) scaled by 8.
-FC1_DRAM_BYTES_PER_LAUNCH = 186.4e6 + 8 * 5.2e6 + 8 * 37.7e6
+# summarised in profiles/cluster_gemm_opt66b_fc1_tokens512.txt: measured at 512 tokens (191.4 MB read,
+# of which 189.5 MB -- packed weights, Wsum, s_w -- do not depend on the token count) with the
+# token-proportional parts (1.94 MB of codes in, 37.75 MB of fp16 output) scaled by 8.
+FC1_DRAM_BYTES_PER_LAUNCH = 189.45e6 + 8 * 1.94e6 + 8 * 37.75e6
 
 
 def _peaks():
