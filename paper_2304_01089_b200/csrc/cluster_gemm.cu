@@ -508,23 +508,41 @@ cluster_gemm_kernel(const Params p)
             }
             cp_async_wait<0>();
         } else {
-        // Activation codes: this thread owns token row `ut` of the tile. A K block of its row is
-        // 16 BITS contiguous bytes, fetched N_A - 1 K blocks ahead with 16-byte cp.async into a slot
-        // that only this thread reads, so no other thread has to be waited for.
+        // Activation codes: this thread owns token row `ut` of the tile and unpacks it. A K block of a
+        // row is 16 BITS contiguous bytes; the rows' K blocks are fetched N_A - 1 K blocks ahead with
+        // 16-byte cp.async into one shared-memory slot per row. The 32 BITS chunks of a warp's 32 rows
+        // are spread over the lanes in memory order (lane l of copy i takes chunk 32 i + l: row
+        // (32 i + l) / BITS of the warp, part (32 i + l) % BITS), so that one warp-wide copy touches
+        // 32 / BITS rows, not 32: the load path looks up one cache line per row touched, and with one
+        // row per lane those look-ups, not the bytes, set the pace. A row's chunks are copied by
+        // lanes of the row owner's own warp, so a __syncwarp after the wait is all the hand-over needs.
         constexpr int N_A = n_a_stages(BITS), PITCH = a_slot_pitch(BITS);
-        const uint32_t a_ring = smem_base + SL.off_a + ut * PITCH;
-        bool a_ok = false;
+        const uint32_t a_ring0 = smem_base + SL.off_a;
+        const uint32_t a_ring = a_ring0 + ut * PITCH;
+        uint32_t d_off[BITS], s_off[BITS];               // where my chunks go in a ring stage / come from in the tile's rows
+        int r_of[BITS];                                  // their rows within the tile
+#pragma unroll
+        for (int i = 0; i < BITS; ++i) {
+            const int c = 32 * i + lane;
+            r_of[i] = (ut & ~31) + c / BITS;
+            d_off[i] = (uint32_t)r_of[i] * PITCH + 16u * (uint32_t)(c % BITS);
+            s_off[i] = (uint32_t)r_of[i] * (uint32_t)p.a_row_bytes + 16u * (uint32_t)(c % BITS);
+        }
+        int rows_left = 0;                               // rows of the tile being fetched that exist
         auto fetch_tile_row = [&]() {
-            const int row = (t_f % p.tiles_m) * (TILE_M * NCTA) + (int)cta_rank * TILE_M + ut;
-            a_ok = row < p.M;
-            a_src = p.a_codes + (int64_t)(a_ok ? row : 0) * p.a_row_bytes;
+            const int row0 = (t_f % p.tiles_m) * (TILE_M * NCTA) + (int)cta_rank * TILE_M;
+            rows_left = p.M - row0;
+            a_src = p.a_codes + (int64_t)(rows_left > 0 ? row0 : 0) * p.a_row_bytes;
         };
         fetch_tile_row();
         auto fetch_next = [&]() {
             if (n_fetched < total_kb) {
-                const uint32_t dst = a_ring + (n_fetched % N_A) * SL.a_stage;
+                const uint32_t dst = a_ring0 + (n_fetched % N_A) * SL.a_stage;
 #pragma unroll
-                for (int j = 0; j < BITS; ++j) cp_async16(dst + 16 * j, a_src + 16 * j, a_ok);
+                for (int i = 0; i < BITS; ++i) {
+                    const bool v = r_of[i] < rows_left;
+                    cp_async16(dst + d_off[i], v ? a_src + s_off[i] : p.a_codes, v);
+                }
                 a_src += 16 * BITS;
                 if (++kb_f == p.n_kb) { kb_f = 0; t_f += n_pairs; fetch_tile_row(); }
             }
@@ -536,7 +554,8 @@ cluster_gemm_kernel(const Params p)
         for (int it = 0; it < total_kb; ++it, ++n_done) {
             const int sp = n_done % N_P, su = n_done % N_U;
             fetch_next();
-            cp_async_wait<N_A - 1>();                    // the group of K block `it` has landed
+            cp_async_wait<N_A - 1>();                    // my copies of K block `it` have landed
+            __syncwarp();                                // ... and those of the lanes that copied my row
             uint32_t pa_w[4][BITS];                      // [unit][word]: unit u of the row is words BITS u ..
             {
                 const uint32_t slot = a_ring + (it % N_A) * SL.a_stage;
