@@ -50,7 +50,8 @@ constexpr int WTILE_BYTES = 8192;                        // one packed weight ti
 constexpr long long WAIT_BUDGET_CYCLES = 4000000000ll;   // about two seconds at the SM clock
 
 __host__ __device__ constexpr int w_rows(int ncta) { return TILE_N / ncta; }           // weight rows staged per CTA
-__host__ __device__ constexpr int n_p_stages(int ncta) { return ncta == 2 ? 4 : 3; }    // packed weight stages
+// packed weight stages; the single-CTA variant (at most 128 tokens) is a weight stream and takes what shared memory is left
+__host__ __device__ constexpr int n_p_stages(int ncta, int bits) { return ncta == 2 ? 4 : (bits == 3 ? 5 : 4); }
 __host__ __device__ constexpr int n_u_stages(int ncta, bool a8) { return ncta == 2 ? (a8 ? 5 : 4) : 2; }   // operand stages
 // ring of packed activation K blocks fetched ahead by the unpack threads: one slot per token row
 // per K block; the pitch is an odd number of 16-byte units so that the threads' vector reads of
@@ -68,7 +69,7 @@ __host__ __device__ constexpr SmemLayout smem_layout(int ncta, int bits, bool a8
     s.p_stage = w_rows(ncta) * KBLK / 2;
     s.a_stage = a8 ? 0 : TILE_M * a_slot_pitch(bits);      // 8-bit activations go straight to the operand stage
     s.off_p = n_u_stages(ncta, a8) * s.u_stage;
-    s.off_a = s.off_p + n_p_stages(ncta) * s.p_stage;
+    s.off_a = s.off_p + n_p_stages(ncta, bits) * s.p_stage;
     s.off_flags = s.off_a + n_a_stages(bits) * s.a_stage;
     s.off_seg_scale = s.off_flags + 2048;
     s.off_seg_buf = s.off_seg_scale + kMaxGemmSegments * 4;
@@ -272,7 +273,7 @@ cluster_gemm_kernel(const Params p)
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     constexpr SmemLayout SL = smem_layout(NCTA, BITS, A8);
     constexpr int W_ROWS = w_rows(NCTA);                 // weight rows this CTA stages and unpacks
-    constexpr int N_P = n_p_stages(NCTA), N_U = n_u_stages(NCTA, A8);
+    constexpr int N_P = n_p_stages(NCTA, BITS), N_U = n_u_stages(NCTA, A8);
     constexpr uint32_t kInstrDesc = instr_desc(NCTA);
     // dynamic shared memory is only guaranteed 16-byte alignment: round up to the swizzle span
     // (the offset is the same in both CTAs of a pair, as cta_group::2 descriptors require)
