@@ -263,8 +263,10 @@ def _oracle_sample(site, rows_ln: int, rows_gemm: int):
     x = workloads.test_tokens(sw, rows_ln)
     n_out = site["n_out"]
     w_packed = site["w"].cpu().numpy() if hasattr(site["w"], "cpu") else site["w"]
-    # the library's position order -> the oracle's contiguous one
-    w_codes = np.ascontiguousarray(oracle.unpack_weights(w_packed, site["L"].K_pad, n_out)[:, np.argsort(site["L"].contiguous_position())])
+    w_codes = oracle.unpack_weights(w_packed, site["L"].K_pad, n_out)
+    if hasattr(site["L"], "contiguous_position"):
+        # weights packed by the library: its position order -> the oracle's contiguous one
+        w_codes = np.ascontiguousarray(w_codes[:, np.argsort(site["L"].contiguous_position())])
     s_w = site["s_w"].cpu().numpy() if hasattr(site["s_w"], "cpu") else site["s_w"]
     wsum = site["wsum"].cpu().numpy() if hasattr(site["wsum"], "cpu") else site["wsum"]
     t0 = time.perf_counter()
