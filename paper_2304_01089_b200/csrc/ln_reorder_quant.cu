@@ -186,8 +186,8 @@ ln_reorder_quant_kernel(const LnParams p)
         // the other operand puts the sums of squares of those rows on a diagonal. One shared-memory
         // instruction and three tensor instructions per 256 values replace some forty conversions
         // and additions per lane. fp16 products are exact in fp32; the variance is
-        // sum(x^2) / C - mean^2, so its relative error grows with (mean / std)^2 (about 1e-6 at
-        // mean = std, 1e-4 at mean = 10 std).
+        // sum(x^2) / C - mean^2, whose relative error grows with (mean / std)^2, so rows whose mean
+        // is more than two standard deviations from zero take a second, centred pass (below).
         const int n_chunks = C >> 3;
         const float inv_C = 1.0f / (float)C;
         const uint32_t zero_s = (uint32_t)__cvta_generic_to_shared(zero16);
@@ -217,7 +217,25 @@ ln_reorder_quant_kernel(const LnParams p)
             const float my_sq = (cq == r ? qa[0] : 0.f) + (cq + 1 == r ? qa[1] : 0.f)     // rows 0-7: D[i][i]
                               + (cq == r ? qb[2] : 0.f) + (cq + 1 == r ? qb[3] : 0.f);    // rows 8-15: D[8 + j][j]
             const float mu = warp_sum(my_sum) * inv_C;
-            const float var = fmaxf(warp_sum(my_sq) * inv_C - mu * mu, 0.f);
+            float var = fmaxf(warp_sum(my_sq) * inv_C - mu * mu, 0.f);
+            if (mu * mu > 4.0f * var) {
+                // The row's mean is more than two standard deviations from zero: sum(x^2)/C - mean^2
+                // cancels too much (relative error ~ 1e-6 (1 + mean^2/var)). Take the centred sum of
+                // squares instead, on the CUDA cores; rows of LayerNorm inputs rarely come here.
+                const uint4* row = reinterpret_cast<const uint4*>(ring + (size_t)d * pitch);
+                const float2 neg_mu = make_float2(-mu, -mu);
+                float2 q2 = make_float2(0.f, 0.f), q2b = make_float2(0.f, 0.f);
+#pragma unroll 2
+                for (int ch = lane; ch < n_chunks; ch += 32) {
+                    const uint4 raw = row[ch];
+                    const __half2* h = reinterpret_cast<const __half2*>(&raw);
+                    const float2 a = add2(__half22float2(h[0]), neg_mu), b = add2(__half22float2(h[1]), neg_mu);
+                    const float2 c = add2(__half22float2(h[2]), neg_mu), e = add2(__half22float2(h[3]), neg_mu);
+                    q2 = fma2(a, a, q2); q2b = fma2(b, b, q2b);
+                    q2 = fma2(c, c, q2); q2b = fma2(e, e, q2b);
+                }
+                var = warp_sum((q2.x + q2.y) + (q2b.x + q2b.y)) * inv_C;
+            }
             const float rstd = 1.0f / sqrtf(var + p.eps);
             if (lane == 0) {
                 stats[d] = make_float2(rstd, -mu * rstd);

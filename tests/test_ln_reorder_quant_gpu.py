@@ -137,6 +137,27 @@ def test_wide_rows_take_the_multi_unit_path_and_zero_tokens_launch_nothing():
     assert bool((codes == CANARY).all())
 
 
+@pytest.mark.parametrize("ratio,bound", [(1.5, 8e-6), (4.0, 8e-6), (32.0, 8e-6)])
+def test_row_mean_far_from_zero(ratio, bound):
+    """The kernel takes the variance as sum(x^2)/C - mean^2 from fp32 sums unless the row's mean is
+    more than two standard deviations from zero (then a centred second pass): LayerNorm outputs
+    against the fp64 oracle on rows whose mean is `ratio` standard deviations away from zero, on both
+    sides of that switch, relative to max|y|."""
+    from paper_2304_01089_b200 import binding
+    rng = np.random.default_rng(int(ratio))
+    C, M, bits = 4096, 64, 4
+    perm, size, scale, zero = random_layout_params(rng, C, 8, bits)
+    L = binding.Layout(perm, size, scale, zero, bits)
+    x = (rng.normal(size=(M, C)) + ratio).astype(np.float16)
+    gm = rng.lognormal(0, 0.3, C).astype(np.float16)
+    bt = rng.normal(size=C).astype(np.float16)
+    _, y_dbg = _run(L, x, gm, bt)
+    y64 = oracle.reorder(oracle.layernorm(x, gm, bt, EPS), perm)
+    err = np.max(np.abs(y_dbg - y64)) / np.abs(y64).max()
+    print(f"mean = {ratio} std: max|dy|/max|y| = {err:.2e}")
+    assert err <= bound
+
+
 def test_non_finite_inputs_still_give_in_range_codes():
     from paper_2304_01089_b200 import binding
     rng = np.random.default_rng(12)
