@@ -94,7 +94,7 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatil
 
 struct LnParams {
     const __half* x; int64_t ldx; const __half* gamma; const __half* beta; float eps;
-    int M, C, n_units, n_stats_warps, depth;
+    int M, C, n_units, n_stats_warps, depth, n_groups;
     const uint16_t* ch_tab;      // [K_pad] channel read for each padded position (pads: any channel, masked later)
     const int32_t* jidx_tab;     // [K_pad] reordered index of each padded position, -1 at pads (debug output)
     const UnitInfo* unit_tab;
@@ -129,7 +129,9 @@ ln_reorder_quant_kernel(const LnParams p)
     volatile int* s_abort = reinterpret_cast<volatile int*>(bars + 3 * D);
     const uint32_t ring_s = (uint32_t)__cvta_generic_to_shared(ring);
     const uint32_t bar_s = (uint32_t)__cvta_generic_to_shared(bars);
-    const int TG = T - 32 * (1 + S), n_gather_warps = TG >> 5;
+    // The gather threads form n_groups groups of TG threads; group j takes rows j, j + n_groups, ...
+    // (narrow layouts leave room for several groups, and a short row is mostly hand-over latency)
+    const int G = p.n_groups, TG = (T - 32 * (1 + S)) / G, n_gather_warps = TG >> 5;
     const int n_rows = (p.M - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;   // rows of this block
 
     if (tid == 0) {
@@ -244,7 +246,7 @@ ln_reorder_quant_kernel(const LnParams p)
         }
     } else {
         // ------------------------------------------------------------ gather warps
-        const int gt = tid - 32 * (1 + S);
+        const int grp = (tid - 32 * (1 + S)) / TG, gt = (tid - 32 * (1 + S)) - grp * TG;
         const bool one_unit = tables_in_regs;              // the fast case: my unit's tables stay in registers
         uint32_t off[32];                                  // byte offset of each source channel in a ring slot
         float2 g2[16], b2[16];                             // gains and biases of source channels 2 i, 2 i + 1
@@ -277,10 +279,10 @@ ln_reorder_quant_kernel(const LnParams p)
         if (one_unit && gt < p.n_units) load_unit(gt, gamma_s, beta_s);
         __syncthreads();
         const float2 magic2 = make_float2(12582912.0f, 12582912.0f);
-        int m = blockIdx.x;
-        int d = 0;
-        uint32_t par = 0;
-        for (int k = 0; k < n_rows; ++k, m += gridDim.x) {
+        int m = (int)blockIdx.x + grp * (int)gridDim.x;
+        int d = grp % D;
+        uint32_t par = (uint32_t)(grp / D) & 1u;
+        for (int k = grp; k < n_rows; k += G, m += G * (int)gridDim.x) {
             mbar_wait<true>(bar_s + 8 * (D + d), par, s_abort, p.status);
             const float2 st = stats[d];
             const float2 rs2 = make_float2(st.x, st.x), nm2 = make_float2(st.y, st.y);
@@ -323,7 +325,8 @@ ln_reorder_quant_kernel(const LnParams p)
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_s + 8 * (2 * D + d));     // this warp has read everything it needs from the slot
-            if (++d == D) { d = 0; par ^= 1u; }
+            d += G;
+            if (d >= D) { d -= D; par ^= 1u; }           // the host keeps n_groups <= depth
         }
     }
 }
@@ -347,7 +350,9 @@ static int planned_blocks(const void* fn, int device, int T, size_t smem, int* b
     std::lock_guard<std::mutex> lock(g_plan_mutex);
     for (const LaunchPlan& pl : g_plans)
         if (pl.fn == fn && pl.device == device && pl.T == T && pl.smem == smem) { *blocks = pl.blocks; return RPTQ_OK; }
-    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return RPTQ_ERR_CUDA;
+    // the attribute belongs to the kernel, not to this plan: always the largest size any plan may ask
+    // for, or a later, smaller plan would take the room away from an earlier one that is cached
+    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess) return RPTQ_ERR_CUDA;
     int n_sm = 0, per_sm = 0;
     if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) return RPTQ_ERR_CUDA;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, T, smem) != cudaSuccess || per_sm < 1) return RPTQ_ERR_CUDA;
@@ -382,15 +387,17 @@ extern "C" int rptq_ln_reorder_quant(const rptq_layout_t* L, const void* x, int6
     depth = depth > 16 ? 16 : depth;
     const size_t smem = (size_t)depth * (pitch + 32) + 64;     // slots, then per slot 8 bytes of statistics and 3 barriers, 16 zero bytes, a flag
 
-    // One gather thread per output unit where that fits beside four statistics warps in a block
-    // of 512 threads (128 registers each); wider layouts get two statistics warps, and beyond 416
+    // One gather thread per output unit where that fits beside four or five statistics warps in a
+    // block of 512 threads (128 registers each), in up to four groups that take alternate rows when
+    // the layout is narrow; wider layouts get two statistics warps, and beyond 416
     // units each gather thread loops over several units and reloads its tables.
     const int want = (L->n_units + 31) / 32 * 32;
-    int TG, S;
-    if (want <= 320) { TG = want; S = 5; }
+    int TG, S, groups = 1;
+    if (want <= 320) { TG = want; S = 5; groups = 320 / TG; groups = groups > 4 ? 4 : groups; }
     else if (want <= 352) { TG = want; S = 4; }
     else { TG = want <= 416 ? want : 416; S = 2; }
-    const int T = 32 * (1 + S) + TG;
+    if (groups > depth) groups = depth;
+    const int T = 32 * (1 + S) + groups * TG;
 
     KernelFn fn = y_dbg ? pick_kernel<true>(L->bits) : pick_kernel<false>(L->bits);
     int blocks = 0;
@@ -399,7 +406,7 @@ extern "C" int rptq_ln_reorder_quant(const rptq_layout_t* L, const void* x, int6
     LnParams p{};
     p.x = static_cast<const __half*>(x); p.ldx = ldx; p.gamma = static_cast<const __half*>(gamma);
     p.beta = static_cast<const __half*>(beta); p.eps = eps; p.M = M; p.C = C; p.n_units = L->n_units;
-    p.n_stats_warps = S; p.depth = depth; p.ch_tab = L->d_src; p.jidx_tab = L->d_jidx; p.unit_tab = L->d_unit;
+    p.n_stats_warps = S; p.depth = depth; p.n_groups = groups; p.ch_tab = L->d_src; p.jidx_tab = L->d_jidx; p.unit_tab = L->d_unit;
     p.codes = static_cast<uint8_t*>(codes); p.row_bytes = L->row_bytes; p.y_dbg = y_dbg; p.status = device_status_word();
     fn<<<M < blocks ? M : blocks, T, smem, static_cast<cudaStream_t>(stream)>>>(p);
     return cudaGetLastError() == cudaSuccess ? RPTQ_OK : RPTQ_ERR_CUDA;

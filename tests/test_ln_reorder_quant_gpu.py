@@ -158,6 +158,24 @@ def test_row_mean_far_from_zero(ratio, bound):
     assert err <= bound
 
 
+def test_wide_then_narrow_then_wide_layouts():
+    """The kernel's launch set-up is cached per shape; a narrow layout (little shared memory) between
+    two uses of a wide one (nearly all of it) must not take the wide one's shared memory away."""
+    from paper_2304_01089_b200 import binding
+    rng = np.random.default_rng(21)
+    cases = []
+    for C in (9216, 256, 9216):
+        perm, size, scale, zero = random_layout_params(rng, C, 6, 4)
+        x = rng.normal(size=(5, C)).astype(np.float16)
+        gm = rng.lognormal(0, 0.3, C).astype(np.float16)
+        bt = rng.normal(size=C).astype(np.float16)
+        L = binding.Layout(perm, size, scale, zero, 4)
+        packed, y_dbg = _run(L, x, gm, bt, want_y=False)
+        packed2, y_dbg = _run(L, x, gm, bt)
+        assert np.array_equal(packed, packed2)
+        _check_against_oracle(x, gm, bt, perm, size, scale, zero, 4, packed2, y_dbg, full_rate=0.999, L=L)
+
+
 def test_non_finite_inputs_still_give_in_range_codes():
     from paper_2304_01089_b200 import binding
     rng = np.random.default_rng(12)
