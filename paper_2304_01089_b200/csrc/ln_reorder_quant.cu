@@ -125,8 +125,8 @@ ln_reorder_quant_kernel(const LnParams p)
     uint8_t* ring = smem_raw;
     float2* stats = reinterpret_cast<float2*>(ring + (size_t)D * pitch);
     uint8_t* zero16 = ring + (size_t)D * pitch + ((8 * (size_t)D + 15) & ~(size_t)15);   // 16 zero bytes, 16-byte aligned
-    uint64_t* bars = reinterpret_cast<uint64_t*>(zero16 + 16);               // landed[D], ready[D], free[D]
-    volatile int* s_abort = reinterpret_cast<volatile int*>(bars + 3 * D);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(zero16 + 16);               // landed[D], ready[D], free[D], tables
+    volatile int* s_abort = reinterpret_cast<volatile int*>(bars + 3 * D + 1);
     const uint32_t ring_s = (uint32_t)__cvta_generic_to_shared(ring);
     const uint32_t bar_s = (uint32_t)__cvta_generic_to_shared(bars);
     // The gather threads form n_groups groups of TG threads; group j takes rows j, j + n_groups, ...
@@ -140,35 +140,41 @@ ln_reorder_quant_kernel(const LnParams p)
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_s + 8 * (D + d)) : "memory");
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar_s + 8 * (2 * D + d)), "r"(n_gather_warps) : "memory");
         }
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar_s + 8 * (3 * D)), "r"(G * n_gather_warps) : "memory");
         *s_abort = 0;
         *reinterpret_cast<uint4*>(zero16) = make_uint4(0u, 0u, 0u, 0u);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    // Gains and biases pass through ring slots 0 and 1 (coalesced loads) so that the gather threads
-    // can pick their own channels' values from shared memory; scattered 2-byte global loads for
-    // 64 values per thread would cost more than a few hundred rows of the kernel proper.
+    // Gains and biases pass through the last two ring slots (coalesced loads) so that the gather
+    // threads can pick their own channels' values from shared memory; scattered 2-byte global loads
+    // for 64 values per thread would cost more than a few hundred rows of the kernel proper. The
+    // producer fills the other slots meanwhile and waits for the `tables` barrier before it reaches
+    // these two.
+    uint8_t* stage_g = ring + (size_t)(D - 2) * pitch;
+    uint8_t* stage_b = ring + (size_t)(D - 1) * pitch;
     {
-        uint4* g_s = reinterpret_cast<uint4*>(ring);
-        uint4* b_s = reinterpret_cast<uint4*>(ring + pitch);
+        uint4* g_s = reinterpret_cast<uint4*>(stage_g);
+        uint4* b_s = reinterpret_cast<uint4*>(stage_b);
         for (int ch = tid; ch < (C >> 3); ch += T) {
             g_s[ch] = __ldg(reinterpret_cast<const uint4*>(p.gamma) + ch);
             b_s[ch] = __ldg(reinterpret_cast<const uint4*>(p.beta) + ch);
         }
     }
     __syncthreads();
-    const __half* gamma_s = reinterpret_cast<const __half*>(ring);
-    const __half* beta_s = reinterpret_cast<const __half*>(ring + pitch);
+    const __half* gamma_s = reinterpret_cast<const __half*>(stage_g);
+    const __half* beta_s = reinterpret_cast<const __half*>(stage_b);
     const bool tables_in_regs = p.n_units <= TG;       // else the gather threads reload tables per unit, from global memory
 
     if (warp == 0) {
         // ------------------------------------------------------------ producer
-        __syncthreads();                     // the gather threads have taken their gains and biases out of the ring
         if (lane == 0) {
             const int64_t row_step = (int64_t)gridDim.x * p.ldx;
             const __half* src = p.x + (int64_t)blockIdx.x * p.ldx;
             int d = 0;
             uint32_t par = 1;                // parity to wait for on free[d]: passes at once the first time round
             for (int k = 0; k < n_rows; ++k) {
+                // the gather threads have taken their gains and biases out of the last two slots
+                if (k == D - 2) mbar_wait(bar_s + 8 * (3 * D), 0u, s_abort, p.status);
                 mbar_wait(bar_s + 8 * (2 * D + d), par, s_abort, p.status);
                 asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_s + 8 * d), "r"(row_bytes_in) : "memory");
                 asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
@@ -181,7 +187,6 @@ ln_reorder_quant_kernel(const LnParams p)
         }
     } else if (warp <= S) {
         // ------------------------------------------------------------ statistics warps
-        __syncthreads();
         // Sum and sum of squares of the row on the tensor cores (mma.sync m16n8k16, fp16 inputs, fp32
         // accumulators): 32 chunks of 8 values are one 16 x 16 operand A, whatever their arrangement;
         // A times a matrix of ones accumulates the sum, and A times its own upper (lower) eight rows as
@@ -251,7 +256,9 @@ ln_reorder_quant_kernel(const LnParams p)
         uint32_t off[32];                                  // byte offset of each source channel in a ring slot
         float2 g2[16], b2[16];                             // gains and biases of source channels 2 i, 2 i + 1
         UnitInfo ui = {1.0f, 0, 0, 0};
-        uint32_t keep[BITS];                               // packed words with all bits set at the unit's real positions
+        // packed words with all bits set at the unit's real positions (8-bit codes: the count of real
+        // positions is enough, a byte mask per word is made on the spot for the few units that have pads)
+        uint32_t keep[BITS == 8 ? 1 : BITS];
         const int qmax = (1 << BITS) - 1;
         auto load_unit = [&](int u, const __half* gamma, const __half* beta) {
             const uint4* sp = reinterpret_cast<const uint4*>(p.ch_tab + u * 32);
@@ -271,13 +278,18 @@ ln_reorder_quant_kernel(const LnParams p)
             const uint4 t4 = __ldg(reinterpret_cast<const uint4*>(p.unit_tab + u));
             ui.inv_s = __uint_as_float(t4.x); ui.zc = (int)t4.y; ui.j0 = (int)t4.z; ui.nvalid = (int)t4.w;
             // pad positions read some real channel (the layout picks one that costs no bank conflict); their codes are masked to 0
-            uint32_t full[32];
+            if constexpr (BITS == 8) {
+                keep[0] = (uint32_t)ui.nvalid;
+            } else {
+                uint32_t full[32];
 #pragma unroll
-            for (int e = 0; e < 32; ++e) full[e] = e < ui.nvalid ? (uint32_t)qmax : 0u;
-            pack32<BITS>(full, keep);
+                for (int e = 0; e < 32; ++e) full[e] = e < ui.nvalid ? (uint32_t)qmax : 0u;
+                pack32<BITS>(full, keep);
+            }
         };
         if (one_unit && gt < p.n_units) load_unit(gt, gamma_s, beta_s);
-        __syncthreads();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_s + 8 * (3 * D));
         const float2 magic2 = make_float2(12582912.0f, 12582912.0f);
         int m = (int)blockIdx.x + grp * (int)gridDim.x;
         int d = grp % D;
@@ -310,8 +322,18 @@ ln_reorder_quant_kernel(const LnParams p)
                 }
                 uint32_t w[BITS];
                 pack32_sat<BITS>(q, w);      // clamps to [0, 2^BITS - 1] and packs
+                if constexpr (BITS == 8) {
+                    if (keep[0] < 32u) {
 #pragma unroll
-                for (int i = 0; i < BITS; ++i) w[i] &= keep[i];
+                        for (int i = 0; i < 8; ++i) {
+                            const int nb = (int)keep[0] - 4 * i;          // real bytes in word i
+                            w[i] &= nb >= 4 ? 0xFFFFFFFFu : nb <= 0 ? 0u : (1u << (8 * nb)) - 1u;
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < BITS; ++i) w[i] &= keep[i];
+                }
                 if constexpr (BITS == 8) {
                     uint4* dst = reinterpret_cast<uint4*>(out_row + u * 32);
                     dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
