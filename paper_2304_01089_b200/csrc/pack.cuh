@@ -42,7 +42,7 @@ __device__ __forceinline__ void pack32(const uint32_t (&q)[32], uint32_t (&w)[BI
 
 // The same words from UNCLAMPED integers: the saturating pack instruction clamps to [0, 15] (or
 // [0, 255]) and appends two codes per instruction, d = (c << 8) | (sat(a) << 4) | sat(b) for 4-bit
-// fields and d = (c << 16) | (sat(a) << 8) | sat(b) for bytes; 3-bit codes take one min first.
+// fields and d = (c << 16) | (sat(a) << 8) | sat(b) for bytes; 3-bit codes are clamped to 7 afterwards.
 __device__ __forceinline__ uint32_t sat_pack_u4(int a, int b, uint32_t c)
 {
     uint32_t d;
@@ -63,7 +63,7 @@ __device__ __forceinline__ uint32_t sat_nibble_word(const int* v)     // 8 integ
     return sat_pack_u4(v[4], v[0], d);
 }
 template <int BITS>
-__device__ __forceinline__ void pack32_sat(int (&v)[32], uint32_t (&w)[BITS])
+__device__ __forceinline__ void pack32_sat(const int (&v)[32], uint32_t (&w)[BITS])
 {
     if constexpr (BITS == 8) {
 #pragma unroll
@@ -72,11 +72,11 @@ __device__ __forceinline__ void pack32_sat(int (&v)[32], uint32_t (&w)[BITS])
 #pragma unroll
         for (int i = 0; i < 4; ++i) w[i] = sat_nibble_word(v + 8 * i);
     } else {
+        // the pack instruction clamps to [0, 15]; nibbles above 7 (bit 3 set) become 7, eight at a time
+        auto clamp7 = [](uint32_t x) { return (x | (((x >> 3) & 0x11111111u) * 7u)) & 0x77777777u; };
+        const uint32_t tail = clamp7(sat_nibble_word(v + 24));
 #pragma unroll
-        for (int e = 0; e < 32; ++e) v[e] = min(v[e], 7);
-        const uint32_t tail = sat_nibble_word(v + 24);
-#pragma unroll
-        for (int j = 0; j < 3; ++j) w[j] = sat_nibble_word(v + 8 * j) | (((tail >> j) & 0x11111111u) << 3);
+        for (int j = 0; j < 3; ++j) w[j] = clamp7(sat_nibble_word(v + 8 * j)) | (((tail >> j) & 0x11111111u) << 3);
     }
 }
 
