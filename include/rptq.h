@@ -14,7 +14,7 @@
  *   - "dev" pointers are device global memory of the device that was current when the layout
  *     was created; "host" pointers are ordinary host memory. The caller owns every buffer. The
  *     library allocates device memory only inside rptq_layout_create (small tables) and for one
- *     lazily created status word per process.
+ *     lazily created status word per device.
  *   - Kernel launches are asynchronous on `stream` (a cudaStream_t passed as void*; NULL is the
  *     default stream). A layout handle is immutable after creation and may be used from several
  *     streams at once.
@@ -118,8 +118,8 @@ int rptq_layout_padded_index(const rptq_layout_t* L, int32_t* padded_index);
 int rptq_layout_destroy(rptq_layout_t* L);
 
 /*
- * Sec. 4.2 "we fuse the reorder operation into the layer norm operation", followed by the
- * cluster quantiser of the Appendix, X~_q,c = Q_k(X~_c, s_c, z_c) with Q_k of Eq. 1:
+ * Sec. 4.2: LayerNorm with the channel reorder fused into its write, followed by the cluster
+ * quantiser of the Appendix, X~_q,c = Q_k(X~_c, s_c, z_c) with Q_k of Eq. 1:
  *   mu = mean_c x[m][c], var = mean_c (x[m][c]-mu)^2, y[c] = (x[m][c]-mu)/sqrt(var+eps)*gamma[c]+beta[c]
  *   (fp32 arithmetic on fp16 inputs), then for reordered position j in cluster c
  *   q = clamp(rne(y[S_j] / s_c) + z_c, 0, 2^bits - 1)
@@ -136,9 +136,9 @@ int rptq_ln_reorder_quant(const rptq_layout_t* L, const void* x, int64_t ldx, co
                           const void* beta, float eps, int M, void* codes, float* y_dbg, void* stream);
 
 /*
- * Sec. 4.2: "We reorder the columns of the weight matrix (dimension C1) based on the input
- * activation reorder index, and the rows (dimension C2) based on the output activation reorder
- * index"; done once before deployment, on the host. W_host is fp32 [N][C] in the [out][in]
+ * Sec. 4.2: the weight's columns (dimension C1, input channels) follow the reorder index of the
+ * site that feeds the layer, its rows (dimension C2, output channels) the index of the site that
+ * reads its output; done once before deployment, on the host. W_host is fp32 [N][C] in the [out][in]
  * orientation (Y = X W^T). Weights are quantised round-to-nearest, symmetric, one scale per output
  * channel (the paper uses GPTQ, which needs a trained model's statistics):
  *   s_w[n] = max_k |W[n][k]| / 7 (1 if the row is zero), w_q = clamp(rne(W / s_w), -8, 7), in fp32.
@@ -174,6 +174,8 @@ int rptq_weight_pack(const rptq_layout_t* Lin, const float* W_host, int N, const
  *            padded position n of Lout's layout; y receives M rows of Lout.row_bytes bytes of
  *            packed codes q' = clamp(rne(v / s'_c') + z'_c'), pad positions 0; ldy is ignored.
  *   Lout     NULL unless y_dtype == RPTQ_OUT_CODES
+ * Limits: Lin.g <= 1024 and Lin.K_pad <= 65536 (the kernel keeps the per-cluster tables in shared
+ * memory); beyond them RPTQ_ERR_UNSUPPORTED.
  */
 int rptq_cluster_gemm(const rptq_layout_t* Lin, const void* a_codes, int M, const void* w_codes,
                       const float* s_w, const int32_t* wsum, int64_t ld_w, const void* bias, int N,
@@ -218,7 +220,7 @@ int rptq_cluster_gemm_debug_acc(const rptq_layout_t* Lin, const void* a_codes, i
                                 const void* w_codes, int N, int m0, int m1, int n0, int n1,
                                 int32_t* acc, void* stream);
 
-/* Host-side readers of the packed formats (format version 1): one byte per code out. */
+/* Host-side readers of the packed formats (format version 2): one byte per code out. */
 int rptq_codes_unpack_host(int K_pad, int bits, const void* packed_host, int64_t M, uint8_t* codes_host);
 int rptq_codes_pack_host(int K_pad, int bits, const uint8_t* codes_host, int64_t M, void* packed_host);
 int rptq_weight_unpack_host(int K_pad, const void* packed_host, int64_t N, int8_t* w_host);
@@ -227,7 +229,8 @@ int64_t rptq_weight_codes_bytes(int K_pad, int64_t N_pad);
 /*
  * Kernels never spin without a limit: a wait that runs out records RPTQ_ERR_DEVICE_TIMEOUT in a
  * device status word, lets the block drain and return, and leaves the output undefined. This call
- * synchronises the device, returns the word in *status (RPTQ_OK if nothing happened) and clears it.
+ * synchronises the current device, returns that device's word in *status (RPTQ_OK if nothing
+ * happened) and clears it. Each device has its own word.
  */
 int rptq_get_device_status(int* status);
 

@@ -12,19 +12,24 @@
 
 namespace rptq {
 
+// One status word per device, allocated on first use with that device current: a kernel that gives
+// up a wait writes to the word of the device it runs on.
+constexpr int kMaxDevices = 64;
 static std::mutex g_status_mutex;
-static int* g_status_word = nullptr;
+static int* g_status_word[kMaxDevices] = {};
 
 int* device_status_word()
 {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
     std::lock_guard<std::mutex> lock(g_status_mutex);
-    if (g_status_word == nullptr) {
+    if (g_status_word[dev] == nullptr) {
         int* p = nullptr;
         if (cudaMalloc(&p, 256) != cudaSuccess) return nullptr;
         if (cudaMemset(p, 0, 256) != cudaSuccess) { cudaFree(p); return nullptr; }
-        g_status_word = p;
+        g_status_word[dev] = p;
     }
-    return g_status_word;
+    return g_status_word[dev];
 }
 
 template <class T>
@@ -390,7 +395,7 @@ int rptq_weight_pack(const rptq_layout_t* Lin, const float* W_host, int N, const
     const int n_kb = K_pad / 128;
     const int rows_stored = (N_pad + 127) / 128 * 128;        // the last tile is filled with zero rows
     uint8_t* packed = static_cast<uint8_t*>(w_codes_host);
-    int failed = 0;
+    int failed = 0;            // set by any worker that meets a non-finite weight (atomic write)
 #pragma omp parallel
     {
         std::vector<uint8_t> row((size_t)K_pad), row_packed((size_t)K_pad / 2);
@@ -407,7 +412,10 @@ int rptq_weight_pack(const rptq_layout_t* Lin, const float* W_host, int N, const
                 const float* w = W_host + (int64_t)src_row * C;
                 float amax = 0.0f;
                 for (int k = 0; k < C; ++k) amax = fmaxf(amax, fabsf(w[k]));
-                if (!std::isfinite(amax)) failed = 1;
+                if (!std::isfinite(amax)) {
+#pragma omp atomic write
+                    failed = 1;
+                }
                 if (amax > 0.0f) s = amax / 7.0f;
                 int j = 0;
                 for (int c = 0; c < g; ++c) {

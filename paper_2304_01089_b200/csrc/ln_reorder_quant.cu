@@ -1,12 +1,23 @@
 // rptq_ln_reorder_quant: LayerNorm with the channel reorder fused in (Sec. 4.2), followed by the
 // per-cluster quantiser (Eq. 1 applied per cluster, Appendix) and packed stores.
 //
-// The paper scatters on write ("the write address is additionally offset based on the reorder
-// index"). Packed sub-byte codes need whole words written at once, so here every thread gathers the
+// The paper scatters on write (Sec. 4.2: LayerNorm's write address carries the reorder index).
+// Packed sub-byte codes need whole words written at once, so here every thread gathers the
 // 32 channels of one output unit (32 consecutive padded positions, always inside one cluster)
 // straight from the raw fp16 row in shared memory, normalises them with the row's statistics and
 // its own channels' gains and biases (held in registers across rows), quantises them with the
 // cluster's parameters and stores 12/16/32 contiguous bytes.
+//
+// The quantiser decision (Eq. 1: round(x / s) + z, clamped) costs one fused multiply-add and half a
+// saturating pack instruction per element. The LayerNorm output is carried scaled by 2^-100 (gains
+// and biases are scaled once per launch; exact), the reciprocal step by 2^-49, the zero point by
+// 2^-149: t = fma(y 2^-100, 2^-49 / s, z 2^-149) is then a multiple of the smallest subnormal, the
+// sum is rounded once, half to even, at exactly the integer grid of y / s + z, and the bit pattern
+// of t IS the integer rne(y / s) + z for every result in [0, 2^24) -- larger results keep their
+// order, negative ones have the sign bit set, so the saturating pack clamps every finite input to
+// the right end. Adding z before the rounding moves exact ties only when z is odd; units with an odd
+// zero point therefore compute the mirrored code qmax - q = clamp(rne(-y / s) + (qmax - z)) (the offset
+// is even again) and flip the packed bits afterwards.
 //
 // Memory-bound by design. A block is persistent over rows. Rows arrive through a ring of
 // shared-memory slots that the copy engine fills many rows ahead; a few warps compute each row's
@@ -37,13 +48,6 @@ __device__ __forceinline__ float2 add2(float2 a, float2 b)
         : "l"(reinterpret_cast<uint64_t&>(a)), "l"(reinterpret_cast<uint64_t&>(b)));
     return d;
 }
-__device__ __forceinline__ float2 mul2(float2 a, float2 b)
-{
-    float2 d;
-    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(reinterpret_cast<uint64_t&>(d))
-        : "l"(reinterpret_cast<uint64_t&>(a)), "l"(reinterpret_cast<uint64_t&>(b)));
-    return d;
-}
 __device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c)
 {
     float2 d;
@@ -62,27 +66,36 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
+// The same test, but the warp may stay suspended in the instruction for up to `ns` nanoseconds
+// while the phase has not completed (it wakes up when it does).
+__device__ __forceinline__ bool mbar_try_wait_for(uint32_t bar, uint32_t parity, uint32_t ns)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity), "r"(ns) : "memory");
+    return ok != 0;
+}
 __device__ __forceinline__ void mbar_arrive(uint32_t bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 constexpr long long kLnWaitBudgetCycles = 4000000000ll;   // about two seconds at the SM clock
 
-// Bounded wait. When the budget runs out the status word is set, every later wait in the block
+// Bounded wait. A warp that has to wait sleeps inside the barrier instruction (a few microseconds
+// at a time) instead of polling: the waiting roles would otherwise take a fifth of the block's
+// issue slots. When the budget runs out the status word is set, every later wait in the block
 // returns at once, and the caller carries on with whatever the slot holds: the loops have fixed
 // trip counts, so the kernel still ends.
-template <bool BACK_OFF = false>
 __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status)
 {
     if (mbar_try_wait(bar, parity)) return;
     const long long t0 = clock64();
 #pragma unroll 1
     while (true) {
-#pragma unroll 1
-        for (int i = 0; i < 256; ++i) {
-            if (mbar_try_wait(bar, parity)) return;
-            if constexpr (BACK_OFF) __nanosleep(200);    // many warps wait here: leave the issue slots to the others
-        }
+        if (mbar_try_wait_for(bar, parity, 4000u)) return;
         if (*abort_flag) return;
         if (clock64() - t0 > kLnWaitBudgetCycles) {
             *abort_flag = 1;
@@ -104,12 +117,14 @@ struct LnParams {
 // Warp roles:
 //   warp 0                 lane 0 keeps the ring full: one contiguous cp.async.bulk per row (at 18-24 KB
 //                          a row, a few rows in flight per SM would leave HBM idle most of the time)
-//   warps 1 .. S           statistics: a warp takes every S-th row, reads it twice from shared memory
-//                          (mean, then the sum of squared deviations) and publishes (rstd, -mean * rstd)
+//   warps 1 .. S           statistics: a warp takes every S-th row, forms the sum and the sum of squares on
+//                          the tensor cores (a centred second pass only for rows whose mean is far from
+//                          zero) and publishes (rstd, -mean * rstd)
 //   the other warps        gather: each thread owns one output unit. Its 32 source offsets, gains and
 //                          biases stay in registers across rows; per row it reads its 32 raw fp16
-//                          values, forms y = ((x * rstd - mean * rstd) * gain + bias) in fp32,
-//                          quantises and stores 12/16/32 contiguous bytes
+//                          values, forms y = ((x * rstd - mean * rstd) * gain + bias) in fp32 (three
+//                          fused multiply-adds per element, the last one being the quantiser decision),
+//                          packs and stores 12/16/32 contiguous bytes
 // Per ring slot three mbarriers hand the row over: landed (copy engine) -> ready (statistics) ->
 // free (all gather warps), which lets the producer refill it.
 // DBG adds the optional fp32 output of the reordered LayerNorm values (off the fast path).
@@ -170,20 +185,29 @@ ln_reorder_quant_kernel(const LnParams p)
         if (lane == 0) {
             const int64_t row_step = (int64_t)gridDim.x * p.ldx;
             const __half* src = p.x + (int64_t)blockIdx.x * p.ldx;
-            int d = 0;
+            int d = 0, n_issued = 0;
             uint32_t par = 1;                // parity to wait for on free[d]: passes at once the first time round
             for (int k = 0; k < n_rows; ++k) {
                 // the gather threads have taken their gains and biases out of the last two slots
                 if (k == D - 2) mbar_wait(bar_s + 8 * (3 * D), 0u, s_abort, p.status);
                 mbar_wait(bar_s + 8 * (2 * D + d), par, s_abort, p.status);
+                if (*s_abort) break;         // a wait ran out somewhere in the block: issue nothing more
                 asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_s + 8 * d), "r"(row_bytes_in) : "memory");
                 asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                              ::"r"(ring_s + d * pitch), "l"(src), "r"(row_bytes_in), "r"(bar_s + 8 * d) : "memory");
                 src += row_step;
+                ++n_issued;
                 if (++d == D) { d = 0; par ^= 1u; }
             }
-            // every copy has landed before the block's shared memory goes away: the statistics warps
-            // wait for each of them
+            // Every copy has landed before the block's shared memory goes away. Normally the statistics
+            // warps have waited for each of them; after a give-up they no longer wait, so this lane
+            // does, for the copies that may still be in flight (a bounded number of polls each).
+            if (*s_abort) {
+                for (int i = n_issued > D ? n_issued - D : 0; i < n_issued; ++i) {
+                    const uint32_t b = bar_s + 8 * (i % D), ph = (uint32_t)(i / D) & 1u;
+                    for (int t = 0; t < (1 << 22) && !mbar_try_wait(b, ph); ++t) __nanosleep(64);
+                }
+            }
         }
     } else if (warp <= S) {
         // ------------------------------------------------------------ statistics warps
@@ -204,10 +228,7 @@ ln_reorder_quant_kernel(const LnParams p)
             const uint32_t row_s = ring_s + (uint32_t)d * pitch;
             float cs[4] = {0.f, 0.f, 0.f, 0.f}, qa[4] = {0.f, 0.f, 0.f, 0.f}, qb[4] = {0.f, 0.f, 0.f, 0.f};
             const uint32_t ones = 0x3C003C00u;       // two fp16 ones
-#pragma unroll 2
-            for (int c0 = 0; c0 < n_chunks; c0 += 32) {
-                const int ch = c0 + lane;
-                const uint32_t addr = ch < n_chunks ? row_s + 16u * (uint32_t)ch : zero_s;
+            auto tile = [&](uint32_t addr) {
                 uint32_t a0, a1, a2, a3;
                 asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
                              : "=r"(a0), "=r"(a1), "=r"(a2), "=r"(a3) : "r"(addr));
@@ -217,7 +238,13 @@ ln_reorder_quant_kernel(const LnParams p)
                              : "+f"(qa[0]), "+f"(qa[1]), "+f"(qa[2]), "+f"(qa[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(a0), "r"(a2));
                 asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
                              : "+f"(qb[0]), "+f"(qb[1]), "+f"(qb[2]), "+f"(qb[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(a1), "r"(a3));
-            }
+            };
+            // whole groups of 32 chunks (512 bytes per step), then the ragged end with zeros for the missing chunks
+            const int n_full = n_chunks >> 5;
+            uint32_t addr = row_s + 16u * (uint32_t)lane;
+#pragma unroll 4
+            for (int i = 0; i < n_full; ++i, addr += 512u) tile(addr);
+            if (n_chunks & 31) tile((n_full << 5) + lane < n_chunks ? addr : zero_s);
             // accumulator fragment: c0, c1 = row lane / 4, columns 2 (lane % 4) + {0, 1}; c2, c3 = row lane / 4 + 8
             const int r = lane >> 2, cq = (lane & 3) * 2;
             const float my_sum = (lane & 3) == 0 ? cs[0] + cs[2] : 0.f;                 // column 0 of all 16 rows
@@ -253,13 +280,16 @@ ln_reorder_quant_kernel(const LnParams p)
         // ------------------------------------------------------------ gather warps
         const int grp = (tid - 32 * (1 + S)) / TG, gt = (tid - 32 * (1 + S)) - grp * TG;
         const bool one_unit = tables_in_regs;              // the fast case: my unit's tables stay in registers
-        uint32_t off[32];                                  // byte offset of each source channel in a ring slot
-        float2 g2[16], b2[16];                             // gains and biases of source channels 2 i, 2 i + 1
-        UnitInfo ui = {1.0f, 0, 0, 0};
+        uint32_t off[32];                                  // shared-memory address of each source channel in ring slot 0
+        float2 g2[16], b2[16];                             // gains and biases of source channels 2 i, 2 i + 1, times 2^-100
+        float2 inv_s2 = make_float2(0.f, 0.f), z2 = make_float2(0.f, 0.f);   // +-2^-49 / s_c and the (even) offset times 2^-149, twice
+        uint32_t flip = 0u;                                // all ones when the unit computes the mirrored code
         // packed words with all bits set at the unit's real positions (8-bit codes: the count of real
         // positions is enough, a byte mask per word is made on the spot for the few units that have pads)
         uint32_t keep[BITS == 8 ? 1 : BITS];
-        const int qmax = (1 << BITS) - 1;
+        constexpr int qmax = (1 << BITS) - 1;
+        constexpr float k2m100 = 7.888609052210118e-31f;    // 2^-100
+        constexpr float k2m49 = 1.7763568394002505e-15f;    // 2^-49
         auto load_unit = [&](int u, const __half* gamma, const __half* beta) {
             const uint4* sp = reinterpret_cast<const uint4*>(p.ch_tab + u * 32);
 #pragma unroll
@@ -269,86 +299,97 @@ ln_reorder_quant_kernel(const LnParams p)
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const uint32_t c0 = w[j] & 0xFFFFu, c1 = w[j] >> 16;
-                    off[8 * i + 2 * j] = 2u * c0;
-                    off[8 * i + 2 * j + 1] = 2u * c1;
-                    g2[4 * i + j] = make_float2(__half2float(gamma[c0]), __half2float(gamma[c1]));
-                    b2[4 * i + j] = make_float2(__half2float(beta[c0]), __half2float(beta[c1]));
+                    off[8 * i + 2 * j] = ring_s + 2u * c0;
+                    off[8 * i + 2 * j + 1] = ring_s + 2u * c1;
+                    g2[4 * i + j] = make_float2(__half2float(gamma[c0]) * k2m100, __half2float(gamma[c1]) * k2m100);
+                    b2[4 * i + j] = make_float2(__half2float(beta[c0]) * k2m100, __half2float(beta[c1]) * k2m100);
                 }
             }
             const uint4 t4 = __ldg(reinterpret_cast<const uint4*>(p.unit_tab + u));
-            ui.inv_s = __uint_as_float(t4.x); ui.zc = (int)t4.y; ui.j0 = (int)t4.z; ui.nvalid = (int)t4.w;
+            const int z = (int)t4.y + 0x4B400000, nvalid = (int)t4.w;
+            const bool odd = (z & 1) != 0;
+            const int z_even = odd ? qmax - z : z;
+            const float inv_s_sc = (odd ? -__uint_as_float(t4.x) : __uint_as_float(t4.x)) * k2m49;
+            // z_even * 2^-149: the subnormal whose fraction field is |z_even|
+            const float z_sc = __uint_as_float(z_even >= 0 ? (uint32_t)z_even : (0x80000000u | (uint32_t)(-z_even)));
+            inv_s2 = make_float2(inv_s_sc, inv_s_sc);
+            z2 = make_float2(z_sc, z_sc);
+            flip = odd ? 0xFFFFFFFFu : 0u;
             // pad positions read some real channel (the layout picks one that costs no bank conflict); their codes are masked to 0
             if constexpr (BITS == 8) {
-                keep[0] = (uint32_t)ui.nvalid;
+                keep[0] = (uint32_t)nvalid;
             } else {
                 uint32_t full[32];
 #pragma unroll
-                for (int e = 0; e < 32; ++e) full[e] = e < ui.nvalid ? (uint32_t)qmax : 0u;
+                for (int e = 0; e < 32; ++e) full[e] = e < nvalid ? (uint32_t)qmax : 0u;
                 pack32<BITS>(full, keep);
             }
         };
         if (one_unit && gt < p.n_units) load_unit(gt, gamma_s, beta_s);
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_s + 8 * (3 * D));
-        const float2 magic2 = make_float2(12582912.0f, 12582912.0f);
-        int m = (int)blockIdx.x + grp * (int)gridDim.x;
-        int d = grp % D;
-        uint32_t par = (uint32_t)(grp / D) & 1u;
-        for (int k = grp; k < n_rows; k += G, m += G * (int)gridDim.x) {
-            mbar_wait<true>(bar_s + 8 * (D + d), par, s_abort, p.status);
-            const float2 st = stats[d];
-            const float2 rs2 = make_float2(st.x, st.x), nm2 = make_float2(st.y, st.y);
-            const uint8_t* slot = ring + (size_t)d * pitch;
-            uint8_t* out_row = p.codes + (int64_t)m * p.row_bytes;
-            for (int u = gt; u < p.n_units; u += TG) {
-                if (!one_unit) load_unit(u, p.gamma, p.beta);
-                const float2 inv_s2 = make_float2(ui.inv_s, ui.inv_s);
-                int q[32];                   // rne(y / s) + z, not yet clamped
+        // Every gather thread walks all of the block's rows with counters that do not depend on the
+        // thread (slot, parity, whose turn it is), so the slot's base address is the same value in
+        // every thread of the kernel's view; a group only works on its own rows.
+        int d = 0, turn = 0;
+        uint32_t par = 0;
+        for (int k = 0; k < n_rows; ++k) {
+            if (turn == grp) {
+                mbar_wait(bar_s + 8 * (D + d), par, s_abort, p.status);
+                const float2 st = stats[d];
+                const float2 rs2 = make_float2(st.x, st.x), nm2 = make_float2(st.y, st.y);
+                const uint32_t slot = (uint32_t)d * pitch;
+                const int m = (int)blockIdx.x + k * (int)gridDim.x;
+                uint8_t* out_row = p.codes + (int64_t)m * p.row_bytes;
+                for (int u = gt; u < p.n_units; u += TG) {
+                    if (!one_unit) load_unit(u, p.gamma, p.beta);
+                    int q[32];                   // rne(y / s) + z (or its mirror), not yet clamped
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const __half h0 = *reinterpret_cast<const __half*>(slot + off[2 * i]);
-                    const __half h1 = *reinterpret_cast<const __half*>(slot + off[2 * i + 1]);
-                    const float2 xh = fma2(make_float2(__half2float(h0), __half2float(h1)), rs2, nm2);
-                    const float2 y = fma2(xh, g2[i], b2[i]);
-                    // the quantiser decision of quant_code (pack.cuh), two values at a time
-                    const float2 t = fma2(y, inv_s2, magic2);
-                    q[2 * i] = __float_as_int(t.x) + ui.zc;
-                    q[2 * i + 1] = __float_as_int(t.y) + ui.zc;
-                    if constexpr (DBG) {
-                        const int j0 = __ldg(p.jidx_tab + u * 32 + 2 * i), j1 = __ldg(p.jidx_tab + u * 32 + 2 * i + 1);
-                        if (j0 >= 0) p.y_dbg[(int64_t)m * C + j0] = y.x;
-                        if (j1 >= 0) p.y_dbg[(int64_t)m * C + j1] = y.y;
-                    }
-                }
-                uint32_t w[BITS];
-                pack32_sat<BITS>(q, w);      // clamps to [0, 2^BITS - 1] and packs
-                if constexpr (BITS == 8) {
-                    if (keep[0] < 32u) {
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            const int nb = (int)keep[0] - 4 * i;          // real bytes in word i
-                            w[i] &= nb >= 4 ? 0xFFFFFFFFu : nb <= 0 ? 0u : (1u << (8 * nb)) - 1u;
+                    for (int i = 0; i < 16; ++i) {
+                        uint16_t h0, h1;
+                        asm volatile("ld.shared.u16 %0, [%1];" : "=h"(h0) : "r"(off[2 * i] + slot));
+                        asm volatile("ld.shared.u16 %0, [%1];" : "=h"(h1) : "r"(off[2 * i + 1] + slot));
+                        const float2 xh = fma2(make_float2(__half2float(__ushort_as_half(h0)), __half2float(__ushort_as_half(h1))), rs2, nm2);
+                        const float2 y = fma2(xh, g2[i], b2[i]);             // LayerNorm outputs times 2^-100
+                        const float2 t = fma2(y, inv_s2, z2);                // the integers themselves (see the head of the file)
+                        q[2 * i] = __float_as_int(t.x);
+                        q[2 * i + 1] = __float_as_int(t.y);
+                        if constexpr (DBG) {
+                            const int ja = __ldg(p.jidx_tab + u * 32 + 2 * i), jb = __ldg(p.jidx_tab + u * 32 + 2 * i + 1);
+                            if (ja >= 0) p.y_dbg[(int64_t)m * C + ja] = y.x * 1.2676506002282294e30f;   // times 2^100, exact
+                            if (jb >= 0) p.y_dbg[(int64_t)m * C + jb] = y.y * 1.2676506002282294e30f;
                         }
                     }
-                } else {
+                    uint32_t w[BITS];
+                    pack32_sat<BITS>(q, w, flip);      // clamps to [0, 2^BITS - 1], packs, flips mirrored units
+                    if constexpr (BITS == 8) {
+                        if (keep[0] < 32u) {
 #pragma unroll
-                    for (int i = 0; i < BITS; ++i) w[i] &= keep[i];
+                            for (int i = 0; i < 8; ++i) {
+                                const int nb = (int)keep[0] - 4 * i;          // real bytes in word i
+                                w[i] &= nb >= 4 ? 0xFFFFFFFFu : nb <= 0 ? 0u : (1u << (8 * nb)) - 1u;
+                            }
+                        }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < BITS; ++i) w[i] &= keep[i];
+                    }
+                    if constexpr (BITS == 8) {
+                        uint4* dst = reinterpret_cast<uint4*>(out_row + u * 32);
+                        dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+                        dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+                    } else if constexpr (BITS == 4) {
+                        *reinterpret_cast<uint4*>(out_row + u * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+                    } else {
+                        uint32_t* dst = reinterpret_cast<uint32_t*>(out_row + u * 12);
+                        dst[0] = w[0]; dst[1] = w[1]; dst[2] = w[2];
+                    }
                 }
-                if constexpr (BITS == 8) {
-                    uint4* dst = reinterpret_cast<uint4*>(out_row + u * 32);
-                    dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
-                    dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
-                } else if constexpr (BITS == 4) {
-                    *reinterpret_cast<uint4*>(out_row + u * 16) = make_uint4(w[0], w[1], w[2], w[3]);
-                } else {
-                    uint32_t* dst = reinterpret_cast<uint32_t*>(out_row + u * 12);
-                    dst[0] = w[0]; dst[1] = w[1]; dst[2] = w[2];
-                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_s + 8 * (2 * D + d));     // this warp has read everything it needs from the slot
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_s + 8 * (2 * D + d));     // this warp has read everything it needs from the slot
-            d += G;
-            if (d >= D) { d -= D; par ^= 1u; }           // the host keeps n_groups <= depth
+            if (++d == D) { d = 0; par ^= 1u; }
+            if (++turn == G) turn = 0;
         }
     }
 }

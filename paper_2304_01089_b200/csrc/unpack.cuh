@@ -1,4 +1,4 @@
-// Device-side readers of the packed code formats (format version 1, described in rptq.h).
+// Device-side readers of the packed code formats (format version 2, described in rptq.h).
 // 32 consecutive codes (one contraction step) become eight 32-bit words of four 8-bit operands
 // each, in K order: out[2i] holds codes 8i..8i+3, out[2i+1] codes 8i+4..8i+7.
 #pragma once

@@ -61,7 +61,9 @@ def _ln_codes(site, L, M):
     want_lib = np.ascontiguousarray(want[:, pos])
     got = oracle.unpack(codes[torch.from_numpy(rows).cuda()].cpu().numpy(), L.K_pad, site.bits)
     diff = np.abs(got.astype(int) - want_lib.astype(int))
-    assert diff.max() <= 1 and (diff != 0).mean() <= 1e-4 * (L.K_pad / site.w.hidden) + 2e-4
+    # the benchmark spec's bar for kernel (a) against the fp64 oracle: all within +-1, >= 99.99 % equal (over the
+    # real positions of the sampled rows; pads always agree)
+    assert diff.max() <= 1 and (diff != 0).sum() <= 1e-4 * len(rows) * site.w.hidden
     codes[torch.from_numpy(rows).cuda()] = torch.from_numpy(oracle.pack(want_lib, site.bits)).cuda()
     return codes, rows, want
 
@@ -103,6 +105,28 @@ def test_layernorm_to_linear_full_size(name, li, Ms):
         k = int(np.where(rows == m0)[0][0])
         assert np.array_equal(acc.cpu().numpy()[:, 0, :].astype(np.int64),
                               oracle.cluster_acc(a_rows[k:k + 1], w_codes_o[n_out - 64:], site.cal.size)[:, 0, :])
+        if M >= 4096:
+            # The same accumulators out of the tensor-core path of this very launch shape (persistent
+            # tiles, every K block, both accumulator buffers): the cluster under test gets scale 1 and
+            # every other one a vanishing scale, with s_w = 1, z = 0 and no Wsum, so the fp32 output is
+            # that cluster's integer accumulator. Sampled rows, two column windows, three clusters.
+            order = np.argsort(site.cal.size)
+            picks = [int(order[-1]), int(order[len(order) // 2]), int(order[np.nonzero(site.cal.size[order])[0][0]])]
+            ones = torch.ones(n_out, dtype=torch.float32, device="cuda")
+            zeros_ws = torch.zeros_like(dev["wsum"])
+            cols = np.r_[0:48, n_out - 48:n_out]
+            want_acc = oracle.cluster_acc(a_rows, np.ascontiguousarray(w_codes_o[cols]), site.cal.size)
+            for c in picks:
+                sc = np.full(L.g, 2.0 ** -80, np.float32)
+                sc[c] = 1.0
+                Lc = binding.Layout(site.cal.perm, site.cal.size, sc, np.zeros(L.g, np.int32), site.bits, order=binding.ORDER_INTERLEAVED)
+                assert np.array_equal(Lc.padded_index(), L.padded_index())
+                binding.cluster_gemm(Lc, codes, M, dev["w"], ones, zeros_ws, n_out, y32)
+                torch.cuda.synchronize()
+                assert binding.get_device_status() == 0
+                got_acc = y32[ridx][:, torch.from_numpy(cols).cuda()].cpu().numpy()
+                assert np.array_equal(np.rint(got_acc).astype(np.int64), want_acc[c]) and np.all(np.abs(got_acc - np.rint(got_acc)) < 1e-6), \
+                    f"cluster {c} (n_c = {site.cal.size[c]}) through the tensor-core path"
 
 
 def test_fc1_relu_requantise_fc2_chain_full_size():
@@ -160,7 +184,9 @@ def test_fc1_relu_requantise_fc2_chain_full_size():
     got2 = oracle.unpack(h_codes[ridx].cpu().numpy(), K2, bits2)
     diff = np.abs(got2.astype(int) - want2_lib.astype(int))
     print(f"re-quantised FC1 output: {(diff != 0).mean():.2e} of codes differ from the fp64 oracle, max {diff.max()}")
-    assert diff.max() <= 1 and (diff != 0).mean() <= 3e-4
+    # the epilogue decides from the GEMM's fp32 output, whose error (~1e-6 of max|h|) moves a value
+    # across a rounding boundary with probability ~ 4 * 2^bits * 1e-6: 1e-4 + 2^bits * 4e-6 is the bar
+    assert diff.max() <= 1 and (diff != 0).sum() <= (1e-4 + (1 << bits2) * 4e-6) * len(rows) * H
     assert not got2[:, ~real].any()
     # FC2 at full size with the oracle's codes planted in the sampled rows
     h_codes[ridx] = torch.from_numpy(oracle.pack(want2_lib, bits2)).cuda()
