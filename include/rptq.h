@@ -234,6 +234,19 @@ int64_t rptq_weight_codes_bytes(int K_pad, int64_t N_pad);
  */
 int rptq_get_device_status(int* status);
 
+/*
+ * Measurement aid (the paper has no counterpart): launches, on `stream`, a kernel that issues the
+ * cluster GEMM's own tensor-core instruction -- tcgen05.mma kind::i8 over CTA pairs, 256 x 256 x 32,
+ * unsigned x signed 8-bit into int32 -- back to back on operands resident in shared memory, with no
+ * loads, unpacking or epilogue, on every SM pair of the current device: n_batches batches of 32
+ * instructions per pair. Time the launch with events on `stream`; *ops_out receives the integer
+ * operations it performs (2 * 256 * 256 * 32 per instruction), so ops / time is the int8 tensor
+ * ceiling of this device at the clocks it ran at.
+ *   failed_dev  dev int, zero before the call: set to 1 if a bounded wait inside the kernel ran out
+ *   n_batches   1 .. 2^20 (2000 is a few milliseconds)
+ */
+int rptq_probe_int8_peak(int n_batches, int* failed_dev, double* ops_out, void* stream);
+
 const char* rptq_status_string(int status);
 int rptq_format_version(void);
 

@@ -26,6 +26,7 @@ EXPORTS = (
     "rptq_weight_pack", "rptq_cluster_gemm", "rptq_cluster_gemm_debug_acc", "rptq_codes_unpack_host",
     "rptq_codes_pack_host", "rptq_weight_unpack_host", "rptq_get_device_status", "rptq_status_string",
     "rptq_format_version", "rptq_layout_padded_index", "rptq_weight_codes_bytes", "rptq_cluster_gemm_noalloc",
+    "rptq_probe_int8_peak",
 )
 
 
@@ -55,6 +56,7 @@ def _load(path: str = LIB_PATH) -> C.CDLL:
     lib.rptq_codes_pack_host.argtypes = [i32, i32, vp, i64, vp]
     lib.rptq_weight_unpack_host.argtypes = [i32, vp, i64, vp]
     lib.rptq_weight_codes_bytes.argtypes = [i32, i64]
+    lib.rptq_probe_int8_peak.argtypes = [i32, vp, C.POINTER(C.c_double), vp]
     lib.rptq_get_device_status.argtypes = [C.POINTER(i32)]
     lib.rptq_status_string.argtypes = [i32]
     lib.rptq_status_string.restype = C.c_char_p
@@ -270,6 +272,14 @@ def weight_unpack_host(packed: np.ndarray, k_pad: int, n_rows: int) -> np.ndarra
     out = np.empty((N, k_pad), np.int8)
     _check(_lib.rptq_weight_unpack_host(int(k_pad), _np_ptr(packed), N, _np_ptr(out)), "rptq_weight_unpack_host")
     return out
+
+
+def probe_int8_peak(n_batches: int, failed, stream=None) -> float:
+    """rptq_probe_int8_peak: launches the operand-resident tcgen05.mma kind::i8 loop; returns the
+    integer operations it performs. `failed` is a zeroed int32 device tensor of one element."""
+    ops = C.c_double()
+    _check(_lib.rptq_probe_int8_peak(int(n_batches), _dev_ptr(failed), C.byref(ops), _stream_ptr(stream)), "rptq_probe_int8_peak")
+    return float(ops.value)
 
 
 def get_device_status() -> int:

@@ -19,7 +19,8 @@
 //               fetches the words of its own items with cp.async into a private ring of
 //               shared-memory slots, several K blocks ahead. 8-bit codes need no unpacking: with
 //               CTA pairs they are copied straight into the operand stage (template flag A8)
-//   warp 1      MMA issuer: four tcgen05.mma (K = 32 each) per K block; each cluster accumulates
+//   warp 1      MMA issuer (the whole warp in converged control flow, one elected lane issues):
+//               four tcgen05.mma (K = 32 each) per K block; each cluster accumulates
 //               into one of two 256-column TMEM buffers (the layout's step flags say which) and
 //               is committed at its last step. A cluster's steps need not be adjacent: in the
 //               interleaved unit order a small cluster's step sits between those of a large one,
@@ -45,6 +46,10 @@ constexpr int TILE_M = 128, TILE_N = 256, KBLK = 128;   // TILE_M is per CTA
 constexpr int THREADS = 512;
 constexpr int UNPACK_WARP0 = 4, N_UNPACK_WARPS = 4;
 constexpr int EPI_WARP0 = 8, N_EPI_WARPS = 8;
+// registers per thread after the in-kernel re-partition (the block is launched with 128 each): the
+// producer / MMA-issuer group, the unpack group, the two epilogue groups (128 running sums per thread)
+constexpr int REGS_WG0 = 40, REGS_UNPACK = 88, REGS_EPI = 192;
+static_assert(128 * (REGS_WG0 + REGS_UNPACK + 2 * REGS_EPI) <= 128 * THREADS, "register pool");
 constexpr int A8_BYTES = TILE_M * KBLK;                  // 16 KiB of 8-bit activation operands per stage
 constexpr int WTILE_BYTES = 8192;                        // one packed weight tile: 128 rows x 64 bytes
 constexpr long long WAIT_BUDGET_CYCLES = 4000000000ll;   // about two seconds at the SM clock
@@ -157,6 +162,21 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         if (clock64() - t0 > WAIT_BUDGET_CYCLES) { *abort_flag = 1; return false; }
     }
 }
+// The same wait for a whole warp that must stay converged (the MMA-issuing warp): the lanes vote on
+// every poll, so all of them leave the loop in the same iteration whatever each one saw.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag)
+{
+    if (__any_sync(0xffffffffu, mbar_try_wait(bar, parity))) return true;
+    const long long t0 = clock64();
+#pragma unroll 1
+    while (true) {
+#pragma unroll 1
+        for (int i = 0; i < 1024; ++i)
+            if (__any_sync(0xffffffffu, mbar_try_wait(bar, parity))) return true;
+        const bool give_up = *abort_flag != 0 || clock64() - t0 > WAIT_BUDGET_CYCLES;
+        if (__any_sync(0xffffffffu, give_up)) { *abort_flag = 1; return false; }
+    }
+}
 __device__ __forceinline__ uint32_t cluster_ctarank()
 {
     uint32_t r;
@@ -188,16 +208,27 @@ __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_gr
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// The two tensor-core instructions below are executed by the WHOLE issuing warp in converged
+// control flow; elect.sync picks the one lane that issues. Measured on an operand-resident loop: a
+// tcgen05.mma issued from a branch that a single lane took costs the issuing thread ~120 clocks,
+// one issued this way ~85, against 134 clocks of tensor-pipe time per instruction.
 template <int NCTA>
 __device__ __forceinline__ void tc_commit(uint32_t bar)
 {
     if constexpr (NCTA == 1) {
-        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+        asm volatile(
+            "{\n\t.reg .pred q;\n\t"
+            "elect.sync _|q, 0xffffffff;\n\t"
+            "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+            ::"r"(bar) : "memory");
     } else {
         // arrives on the barrier at this offset in both CTAs of the pair
         const uint16_t mask = 3;
-        asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-                     ::"r"(bar), "h"(mask) : "memory");
+        asm volatile(
+            "{\n\t.reg .pred q;\n\t"
+            "elect.sync _|q, 0xffffffff;\n\t"
+            "@q tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;\n\t}"
+            ::"r"(bar), "h"(mask) : "memory");
     }
 }
 template <int NCTA>
@@ -205,15 +236,17 @@ __device__ __forceinline__ void tc_mma_i8(uint32_t d_tmem, uint64_t a_desc, uint
 {
     if constexpr (NCTA == 1) {
         asm volatile(
-            "{\n\t.reg .pred p;\n\t"
+            "{\n\t.reg .pred p, q;\n\t"
+            "elect.sync _|q, 0xffffffff;\n\t"
             "setp.ne.b32 p, %4, 0;\n\t"
-            "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+            "@q tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
             ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
     } else {
         asm volatile(
-            "{\n\t.reg .pred p;\n\t"
+            "{\n\t.reg .pred p, q;\n\t"
+            "elect.sync _|q, 0xffffffff;\n\t"
             "setp.ne.b32 p, %4, 0;\n\t"
-            "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+            "@q tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t}"
             ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
     }
 }
@@ -334,7 +367,7 @@ cluster_gemm_kernel(const Params p)
     // The register file is re-partitioned by warpgroup (the epilogue holds 128 running sums per
     // thread); each setmaxnreg is executed by the four warps of its group at one place.
     if (warp < UNPACK_WARP0) {
-      asm volatile("setmaxnreg.dec.sync.aligned.u32 24;");
+      asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS_WG0));
       if (warp == 0) {
         // ------------------------------------------------------------ bulk-copy producer
         if (lane == 0) {
@@ -365,8 +398,10 @@ cluster_gemm_kernel(const Params p)
         }
       } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer (first CTA of a pair only)
-        if (lane == 0 && cta_rank == 0) {
-            // This lane is a single thread of dependent instructions, so the loop is kept short:
+        if (cta_rank == 0) {
+            // The whole warp runs this loop in converged control flow (every value in it is the same
+            // in all lanes); one elected lane issues. It is a single stream of dependent
+            // instructions, so the loop is kept short:
             // stage descriptors are built once, a K block's four step flags come as one word, and a
             // block that lies inside one cluster issues its four MMAs without any test.
             // (the loop runs over all K blocks of all of this pair's tiles with one counter: the
@@ -382,7 +417,7 @@ cluster_gemm_kernel(const Params p)
                     const int s = n_kb_done % N_U;
                     kb = kb + 1 == p.n_kb ? 0 : kb + 1;
                     const uint32_t f4_next = flags4[kb];                              // read while waiting
-                    if (!mbar_wait(bar(B_UFULL + s), (n_kb_done / N_U) & 1, s_abort)) { ok = false; break; }
+                    if (!mbar_wait_warp(bar(B_UFULL + s), (n_kb_done / N_U) & 1, s_abort)) { ok = false; break; }
                     tc_fence_after();
                     // the start-address field counts 16-byte units: one stage further, 32 bytes per step;
                     // the weight operand follows the activation operand in the stage
@@ -407,7 +442,7 @@ cluster_gemm_kernel(const Params p)
                             if (f & STEP_SKIP) continue;
                             if (f & STEP_FIRST) {
                                 // the accumulator's previous cluster has been drained
-                                if (!mbar_wait(bar(B_ACCEMPTY + b), ((par >> b) & 1u) ^ 1u, s_abort)) { ok = false; break; }
+                                if (!mbar_wait_warp(bar(B_ACCEMPTY + b), ((par >> b) & 1u) ^ 1u, s_abort)) { ok = false; break; }
                                 tc_fence_after();
                             }
                             tc_mma_i8<NCTA>(d_tmem, ad + 2 * j, wd + 2 * j, kInstrDesc, (f & STEP_FIRST) ? 0u : 1u);
@@ -429,7 +464,7 @@ cluster_gemm_kernel(const Params p)
       }   // warps 2 and 3 only fill the first warpgroup
     } else if (warp < EPI_WARP0) {
         // ------------------------------------------------------------ unpack warps
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 88;");
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS_UNPACK));
         const int ut = tid - UNPACK_WARP0 * 32;      // 0..127
         uint32_t n_done = 0;
         const int total_kb = ((p.n_tiles - pair_id + n_pairs - 1) / n_pairs) * p.n_kb;
@@ -605,7 +640,7 @@ cluster_gemm_kernel(const Params p)
         }
     } else {
         // ------------------------------------------------------------ epilogue warps
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 200;");
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(REGS_EPI));
         const int ew = warp - EPI_WARP0;
         const int q = ew & 3, h = ew >> 2;           // TMEM lane quarter (= warp % 4), column half
         const int et = ew * 32 + lane;               // 0..255: the column whose tile constants I prepare
@@ -755,7 +790,7 @@ static int launch(const Params& p, int n_sm, cudaStream_t st)
     cudaFuncAttributes attr;
     if (cudaFuncGetAttributes(&attr, fn) != cudaSuccess) return RPTQ_ERR_CUDA;
     // the register re-partition inside the kernel (setmaxnreg) assumes this pool; refuse to launch otherwise
-    if (attr.numRegs * THREADS < 24 * 128 + 88 * 128 + 200 * 256) return RPTQ_ERR_UNSUPPORTED;
+    if (attr.numRegs * THREADS < 128 * (REGS_WG0 + REGS_UNPACK + 2 * REGS_EPI)) return RPTQ_ERR_UNSUPPORTED;
     if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return RPTQ_ERR_CUDA;
     const int slots = n_sm / NCTA;
     const int groups = p.n_tiles < slots ? p.n_tiles : slots;
