@@ -246,6 +246,60 @@ def dequant_matmul(a_codes, w_codes, size, scale, zero, s_w) -> np.ndarray:
     return y
 
 
+# ---------------------------------------------------------------- per-cluster asymmetric weights
+def weight_quantize_clustered(W: np.ndarray, perm, size, k: int = 4, n_pad: Optional[int] = None):
+    """Returns (w_codes uint8 [N_pad][K_pad], s_w fp32 [g][N_pad], z_w int32 [g][N_pad], wsum int32 [g][N_pad])."""
+    W = _arr(W, np.float32)
+    perm, size = _arr(perm, np.int32), _arr(size, np.int32)
+    N, Cn = W.shape
+    n_pad = N if n_pad is None else n_pad
+    g = size.shape[0]
+    _, k_pad = segment_offsets(size)
+    w_codes = np.empty((n_pad, k_pad), np.uint8)
+    s_w = np.empty((g, n_pad), np.float32)
+    z_w = np.empty((g, n_pad), np.int32)
+    wsum = np.empty((g, n_pad), np.int32)
+    _lib.orc_weight_quantize_clustered(_p(W), _i64(N), C.c_int(Cn), C.c_int(g), C.c_int(k), _p(perm), _p(size),
+                                       _i64(n_pad), _i32(k_pad), _p(w_codes), _p(s_w), _p(z_w), _p(wsum))
+    return w_codes, s_w, z_w, wsum
+
+
+def code_rowsums(a_codes, size) -> np.ndarray:
+    a_codes, size = _arr(a_codes, np.uint8), _arr(size, np.int32)
+    M, k_pad = a_codes.shape
+    out = np.empty((M, size.shape[0]), np.int32)
+    _lib.orc_code_rowsums(_p(a_codes), _i64(M), _i32(k_pad), C.c_int(size.shape[0]), _p(size), _p(out))
+    return out
+
+
+def _asym_args(a_codes, w_codes, size, scale, zero, s_w, z_w):
+    a_codes, w_codes = _arr(a_codes, np.uint8), _arr(w_codes, np.uint8)
+    size, zero = _arr(size, np.int32), _arr(zero, np.int32)
+    scale, s_w, z_w = _arr(scale, np.float64), _arr(s_w, np.float32), _arr(z_w, np.int32)
+    M, k_pad = a_codes.shape
+    N = w_codes.shape[0]
+    g = size.shape[0]
+    assert w_codes.shape[1] == k_pad and s_w.shape == z_w.shape and s_w.shape[0] == g and s_w.shape[1] >= N
+    return a_codes, w_codes, size, scale, zero, s_w, z_w, M, N, k_pad, g
+
+
+def cluster_gemm_asym(a_codes, w_codes, size, scale, zero, s_w, z_w, bias=None, relu=False) -> np.ndarray:
+    a_codes, w_codes, size, scale, zero, s_w, z_w, M, N, k_pad, g = _asym_args(a_codes, w_codes, size, scale, zero, s_w, z_w)
+    b = None if bias is None else _arr(bias, np.float32)
+    y = np.empty((M, N))
+    _lib.orc_cluster_gemm_asym(_p(a_codes), _i64(M), _p(w_codes), _i64(N), _i32(k_pad), C.c_int(g), _p(size), _p(scale),
+                               _p(zero), _p(s_w), _p(z_w), _i64(s_w.shape[1]), _p(b), C.c_int(1 if relu else 0), _p(y))
+    return y
+
+
+def dequant_matmul_asym(a_codes, w_codes, size, scale, zero, s_w, z_w) -> np.ndarray:
+    a_codes, w_codes, size, scale, zero, s_w, z_w, M, N, k_pad, g = _asym_args(a_codes, w_codes, size, scale, zero, s_w, z_w)
+    y = np.empty((M, N))
+    _lib.orc_dequant_matmul_asym(_p(a_codes), _i64(M), _p(w_codes), _i64(N), _i32(k_pad), C.c_int(g), _p(size), _p(scale),
+                                 _p(zero), _p(s_w), _p(z_w), _i64(s_w.shape[1]), _p(y))
+    return y
+
+
 # ---------------------------------------------------------------- calibration pipeline
 class Calibration(NamedTuple):
     perm: np.ndarray      # int32 [C]  reorder index S

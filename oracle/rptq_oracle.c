@@ -567,3 +567,136 @@ void orc_dequant_matmul(const uint8_t* a_codes, int64_t M, const int8_t* w_codes
         }
     free(seg_off);
 }
+
+/* ------------------------------------------------------------------------------------------ */
+/* Per-cluster asymmetric weight parameters (Appendix, W~_q,i = Q_k(W~_i, s^W_i, z^W_i))       */
+/* ------------------------------------------------------------------------------------------ */
+
+/* Appendix: "for one output channel, each weight cluster is quantised with its own asymmetric
+ * parameters". For output row r and input cluster i the parameters come from the Min-Max method
+ * (Eq. 2, taken literally as for the activations) over the row's weights of that cluster, and the
+ * codes from Eq. 1 re-based to [0, 2^k - 1]. (The paper obtains the codes with GPTQ, which needs a
+ * trained model's Hessians; round-to-nearest is used here.) Everything that decides an integer is
+ * evaluated in IEEE fp32, as in orc_weight_quantize.
+ *   w_codes [N_pad][K_pad] unsigned codes in the padded cluster segments, pad positions 0
+ *   s_w, z_w, wsum [g][N_pad]: scale, zero point (for the re-based codes) and the sum of the codes
+ *   over the real channels of the cluster. Empty clusters and rows r >= N: s = 1, z = 0, sum 0. */
+void orc_weight_quantize_clustered(const float* W, int64_t N, int C, int g, int k, const int32_t* perm,
+                                   const int32_t* size, int64_t N_pad, int32_t K_pad,
+                                   uint8_t* w_codes, float* s_w, int32_t* z_w, int32_t* wsum)
+{
+    int32_t* seg_off = (int32_t*)malloc(sizeof(int32_t) * (g + 1));
+    orc_segment_offsets(size, g, seg_off);
+    memset(w_codes, 0, (size_t)(N_pad * K_pad));
+    const float qmax = (float)((1 << k) - 1);
+    for (int64_t r = 0; r < N_pad; ++r)
+        for (int c = 0; c < g; ++c) {
+            s_w[(int64_t)c * N_pad + r] = 1.0f;
+            z_w[(int64_t)c * N_pad + r] = 0;
+            wsum[(int64_t)c * N_pad + r] = 0;
+        }
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < N; ++r) {
+        const float* wr = W + r * C;
+        int j0 = 0;
+        for (int c = 0; c < g; j0 += size[c], ++c) {
+            if (size[c] == 0) continue;
+            float lo = INFINITY, hi = -INFINITY;
+            for (int i = 0; i < size[c]; ++i) {
+                float v = wr[perm[j0 + i]];
+                if (v < lo) lo = v;
+                if (v > hi) hi = v;
+            }
+            volatile float s = (hi - lo) / (float)(1 << k);           /* Eq. 2, denominator 2^k */
+            if (!(s > 0.0f)) s = 1.0f;
+            volatile float mid = (hi + lo) / (2.0f * s);
+            const int32_t z = (1 << (k - 1)) - (int32_t)rintf(mid);    /* re-based zero point */
+            int32_t acc = 0;
+            for (int i = 0; i < size[c]; ++i) {
+                volatile float t = wr[perm[j0 + i]] / s;
+                float q = rintf(t) + (float)z;                         /* Eq. 1 */
+                if (q < 0.0f) q = 0.0f;
+                if (q > qmax) q = qmax;
+                w_codes[r * K_pad + seg_off[c] + i] = (uint8_t)q;
+                acc += (int32_t)q;
+            }
+            s_w[(int64_t)c * N_pad + r] = s;
+            z_w[(int64_t)c * N_pad + r] = z;
+            wsum[(int64_t)c * N_pad + r] = acc;
+        }
+    }
+    free(seg_off);
+}
+
+/* Sums of the activation codes over the real positions of each cluster, xsum[m][c] = sum_{k in
+ * S^c} X_q[m][k]: the third term of the second method needs them. */
+void orc_code_rowsums(const uint8_t* a_codes, int64_t M, int32_t K_pad, int g, const int32_t* size, int32_t* xsum)
+{
+    int32_t* seg_off = (int32_t*)malloc(sizeof(int32_t) * (g + 1));
+    orc_segment_offsets(size, g, seg_off);
+    for (int64_t m = 0; m < M; ++m)
+        for (int c = 0; c < g; ++c) {
+            int32_t s = 0;
+            for (int p = seg_off[c]; p < seg_off[c] + size[c]; ++p) s += a_codes[m * K_pad + p];
+            xsum[m * g + c] = s;
+        }
+    free(seg_off);
+}
+
+/* Appendix, second method, all four terms (the printed expression omits the sums and the cluster
+ * size; written out for one output element):
+ *   Y_q,i[m][n] = sum_k X_q W_q - z^X_i sum_k W_q - z^W_i[n] sum_k X_q + n_i z^X_i z^W_i[n]
+ *   Y[m][n]     = sum_i s^X_i s^W_i[n] Y_q,i[m][n]                       (clusters ascending)
+ * with every sum over the n_i real channels of cluster i, then + bias[n] and ReLU if asked for. */
+void orc_cluster_gemm_asym(const uint8_t* a_codes, int64_t M, const uint8_t* w_codes, int64_t N,
+                           int32_t K_pad, int g, const int32_t* size, const double* scale,
+                           const int32_t* zero, const float* s_w, const int32_t* z_w, int64_t ld,
+                           const float* bias, int relu, double* y)
+{
+    int32_t* seg_off = (int32_t*)malloc(sizeof(int32_t) * (g + 1));
+    orc_segment_offsets(size, g, seg_off);
+#pragma omp parallel for schedule(static)
+    for (int64_t m = 0; m < M; ++m)
+        for (int64_t n = 0; n < N; ++n) {
+            double total = 0.0;
+            for (int c = 0; c < g; ++c) {
+                int64_t xw = 0, sum_w = 0, sum_x = 0;
+                for (int p = seg_off[c]; p < seg_off[c] + size[c]; ++p) {
+                    const int64_t xq = a_codes[m * K_pad + p], wq = w_codes[n * K_pad + p];
+                    xw += xq * wq;
+                    sum_w += wq;
+                    sum_x += xq;
+                }
+                const int64_t zx = zero[c], zw = z_w[(int64_t)c * ld + n];
+                const int64_t yq = xw - zx * sum_w - zw * sum_x + (int64_t)size[c] * zx * zw;
+                total += scale[c] * (double)s_w[(int64_t)c * ld + n] * (double)yq;
+            }
+            if (bias) total += (double)bias[n];
+            if (relu && total < 0.0) total = 0.0;
+            y[m * N + n] = total;
+        }
+    free(seg_off);
+}
+
+/* Appendix, first method with the same parameters: X^ = s^X_i (X_q - z^X_i), W^ = s^W_i[n] (W_q -
+ * z^W_i[n]), Y = X^ W^T in floating point. The cross-check of orc_cluster_gemm_asym. */
+void orc_dequant_matmul_asym(const uint8_t* a_codes, int64_t M, const uint8_t* w_codes, int64_t N,
+                             int32_t K_pad, int g, const int32_t* size, const double* scale,
+                             const int32_t* zero, const float* s_w, const int32_t* z_w, int64_t ld, double* y)
+{
+    int32_t* seg_off = (int32_t*)malloc(sizeof(int32_t) * (g + 1));
+    orc_segment_offsets(size, g, seg_off);
+#pragma omp parallel for schedule(static)
+    for (int64_t m = 0; m < M; ++m)
+        for (int64_t n = 0; n < N; ++n) {
+            double s = 0.0;
+            for (int c = 0; c < g; ++c)
+                for (int p = seg_off[c]; p < seg_off[c] + size[c]; ++p) {
+                    double xh = scale[c] * ((double)a_codes[m * K_pad + p] - (double)zero[c]);
+                    double wh = (double)s_w[(int64_t)c * ld + n] * ((double)w_codes[n * K_pad + p] - (double)z_w[(int64_t)c * ld + n]);
+                    s += xh * wh;
+                }
+            y[m * N + n] = s;
+        }
+    free(seg_off);
+}

@@ -424,3 +424,127 @@ def test_calibration_pipeline_composes_the_pinned_pieces():
     # one clamped top step that Eq. 2 implies
     codes = oracle.quantize(oracle.reorder(y, cal.perm), cal.size, cal.scale, cal.zero, k)
     assert codes.max() == 15 and codes.min() == 0
+
+
+# ------------------------------------------------------------------ per-cluster asymmetric weights (Appendix)
+def test_asymmetric_hand_worked_examples():
+    n = 0
+    for line in _golden_rows("asym_toy.txt"):
+        kind, fields, want = [p.strip() for p in line.split("|")]
+        if kind == "gemm":
+            f = [float(v) for v in fields.split()]
+            yq0, yq1, y = [float(v) for v in want.split()]
+            size = np.array([2, 2], np.int32)
+            a = np.zeros((1, 128), np.uint8); w = np.zeros((1, 128), np.uint8)
+            a[0, 0:2] = f[2:4]; a[0, 32:34] = f[10:12]
+            w[0, 0:2] = f[6:8]; w[0, 32:34] = f[14:16]
+            scale = np.array([f[0], f[8]]); zero = np.array([f[1], f[9]], np.int32)
+            s_w = np.array([[f[4]], [f[12]]], np.float32); z_w = np.array([[f[5]], [f[13]]], np.int32)
+            assert oracle.cluster_gemm_asym(a, w, size, scale, zero, s_w, z_w)[0, 0] == y
+            assert oracle.dequant_matmul_asym(a, w, size, scale, zero, s_w, z_w)[0, 0] == y
+            # the per-cluster integers, through unit scales on one cluster at a time
+            for c, yq in ((0, yq0), (1, yq1)):
+                sc = np.zeros(2); sc[c] = 1.0
+                assert oracle.cluster_gemm_asym(a, w, size, sc, zero, np.ones((2, 1), np.float32), z_w)[0, 0] == yq
+        else:
+            f = fields.split()
+            k, ws = int(f[0]), np.array([float(v) for v in f[1:]], np.float32)
+            wv = want.split()
+            W = np.zeros((1, 8), np.float32); W[0, :3] = ws
+            # the three weights are one cluster, the other five channels another one
+            codes, s_w, z_w, wsum = oracle.weight_quantize_clustered(W, np.arange(8), np.array([3, 5], np.int32), k)
+            assert s_w[0, 0] == np.float32(float(wv[0])) and z_w[0, 0] == int(wv[1])
+            assert codes[0, :3].tolist() == [int(v) for v in wv[2:]] and wsum[0, 0] == sum(int(v) for v in wv[2:])
+            # the other cluster is all zeros: max == min, so s = 1, z = 2^(k-1) and every code equals z
+            assert s_w[1, 0] == 1.0 and z_w[1, 0] == 1 << (k - 1) and np.all(codes[0, 32:37] == 1 << (k - 1))
+        n += 1
+    assert n == 3
+
+
+def _asym_case(seed, M=5, N=7, C=96, g=4, k=4, bits=4):
+    r = _rng(seed)
+    perm = r.permutation(C).astype(np.int32)
+    cuts = np.sort(r.integers(0, C + 1, size=g - 1))
+    size = np.diff(np.concatenate([[0], cuts, [C]])).astype(np.int32)
+    W = (r.normal(size=(N, C)) * r.lognormal(0, 1, size=C)).astype(np.float32)
+    codes_w, s_w, z_w, wsum = oracle.weight_quantize_clustered(W, perm, size, k)
+    off, k_pad = oracle.segment_offsets(size)
+    a = np.zeros((M, k_pad), np.uint8)
+    for c in range(g):
+        a[:, off[c]:off[c] + size[c]] = r.integers(0, 1 << bits, size=(M, size[c]))
+    scale = r.uniform(0.05, 1.5, g)
+    zero = r.integers(-3, 1 << bits, g).astype(np.int32)
+    return dict(perm=perm, size=size, W=W, w=codes_w, s_w=s_w, z_w=z_w, wsum=wsum, a=a, scale=scale, zero=zero, off=off, k_pad=k_pad, k=k)
+
+
+def test_clustered_weight_quantiser_against_a_plain_restatement():
+    for seed, k in ((1, 4), (2, 3), (3, 8)):
+        c = _asym_case(seed, k=k)
+        qmax = (1 << k) - 1
+        j = 0
+        for ci, n_c in enumerate(c["size"]):
+            ch = c["perm"][j:j + n_c]; j += n_c
+            if n_c == 0:
+                assert np.all(c["s_w"][ci] == 1) and not c["z_w"][ci].any() and not c["wsum"][ci].any()
+                continue
+            for n in range(c["W"].shape[0]):
+                w = c["W"][n, ch]
+                s = np.float32(w.max() - w.min()) / np.float32(1 << k)
+                s = s if s > 0 else np.float32(1)
+                z = (1 << (k - 1)) - int(np.rint(np.float32(w.max() + w.min()) / (np.float32(2) * s)))
+                q = np.clip(np.rint(w / s) + z, 0, qmax).astype(np.uint8)
+                got = c["w"][n, c["off"][ci]:c["off"][ci] + n_c]
+                assert c["s_w"][ci, n] == s and c["z_w"][ci, n] == z
+                assert np.array_equal(got, q) and c["wsum"][ci, n] == int(q.sum())
+                # Eq. 2's consequences: the minimum maps to code 0; inside the range the error is at most half a step
+                assert got[np.argmin(w)] == 0
+                err = np.abs(s * (got.astype(np.float64) - z) - w)
+                inside = np.rint(w / s) + z <= qmax
+                assert np.all(err[inside] <= 0.5 * s * (1 + 1e-5))
+        assert not c["w"][:, np.setdiff1d(np.arange(c["k_pad"]), np.concatenate([np.arange(o, o + n) for o, n in zip(c["off"], c["size"])]))].any()
+
+
+def test_asymmetric_integer_method_equals_dequantise_then_matmul():
+    for seed in (11, 12, 13):
+        c = _asym_case(seed, M=6, N=9, C=160, g=5)
+        y2 = oracle.cluster_gemm_asym(c["a"], c["w"], c["size"], c["scale"], c["zero"], c["s_w"], c["z_w"])
+        y1 = oracle.dequant_matmul_asym(c["a"], c["w"], c["size"], c["scale"], c["zero"], c["s_w"], c["z_w"])
+        assert np.max(np.abs(y1 - y2)) <= 1e-12 * np.abs(y1).max()
+        # and a library matmul on the de-quantised operands (contiguous real positions)
+        xh = np.zeros(c["a"].shape); wh = np.zeros(c["w"].shape)
+        for ci, (o, n_c) in enumerate(zip(c["off"], c["size"])):
+            xh[:, o:o + n_c] = c["scale"][ci] * (c["a"][:, o:o + n_c].astype(np.float64) - c["zero"][ci])
+            wh[:, o:o + n_c] = c["s_w"][ci][:, None].astype(np.float64) * (c["w"][:, o:o + n_c].astype(np.float64) - c["z_w"][ci][:, None])
+        assert np.max(np.abs(xh @ wh.T - y2)) <= 1e-12 * np.abs(y2).max()
+        # bias and ReLU
+        b = _rng(seed).normal(size=9).astype(np.float32)
+        yb = oracle.cluster_gemm_asym(c["a"], c["w"], c["size"], c["scale"], c["zero"], c["s_w"], c["z_w"], bias=b, relu=True)
+        assert np.allclose(yb, np.maximum(y2 + b, 0), rtol=0, atol=1e-12 * np.abs(y2).max())
+
+
+def test_asymmetric_method_reduces_to_the_symmetric_one():
+    """z^W = const and s^W_i the same for every cluster: the four-term expression must give what the
+    symmetric path gives on the same integers (codes shifted by 8)."""
+    r = _rng(21)
+    C, N, M, g = 128, 6, 4, 3
+    perm = r.permutation(C).astype(np.int32)
+    size = np.array([50, 0, 78], np.int32)
+    W = (r.normal(size=(N, C)) * 0.02).astype(np.float32)
+    w_sym, s_w, wsum = oracle.weight_quantize(W, perm, size)
+    off, k_pad = oracle.segment_offsets(size)
+    a = np.zeros((M, k_pad), np.uint8)
+    for c in range(g):
+        a[:, off[c]:off[c] + size[c]] = r.integers(0, 16, size=(M, size[c]))
+    scale = r.uniform(0.1, 1, g); zero = r.integers(0, 16, g).astype(np.int32)
+    want = oracle.cluster_gemm(a, w_sym, size, scale, zero, s_w, wsum)
+    w_u = (w_sym.astype(np.int16) + 8).astype(np.uint8)
+    got = oracle.cluster_gemm_asym(a, w_u, size, scale, zero, np.tile(s_w, (g, 1)), np.full((g, N), 8, np.int32))
+    assert np.max(np.abs(got - want)) <= 1e-12 * np.abs(want).max()
+
+
+def test_code_rowsums_brute_force():
+    c = _asym_case(31, M=9, C=200, g=6)
+    got = oracle.code_rowsums(c["a"], c["size"])
+    for m in range(9):
+        for ci, (o, n_c) in enumerate(zip(c["off"], c["size"])):
+            assert got[m, ci] == sum(int(v) for v in c["a"][m, o:o + n_c])

@@ -54,11 +54,43 @@ def test_two_calls_in_a_row_match_the_allocating_entry_point():
         y_new = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
         binding.cluster_gemm_noalloc(dev["L"], dev["a"], M, dev["w"], dev["s_w"], dev["wsum"], N, y_new, bias=dev["bias"])
         torch.cuda.synchronize()
+        # a further call changes nothing in how much device memory is free: the driver's own count,
+        # taken around the call with every buffer already in place
+        free_before, _ = torch.cuda.mem_get_info()
+        binding.cluster_gemm_noalloc(dev["L"], dev["a"], M, dev["w"], dev["s_w"], dev["wsum"], N, y_new, bias=dev["bias"])
+        torch.cuda.synchronize()
+        free_after, _ = torch.cuda.mem_get_info()
+        assert free_after == free_before
         ref, new = y_ref.cpu().numpy(), y_new.cpu().numpy()
         scale = np.abs(want).max()
         assert np.max(np.abs(new - ref)) <= TOL * scale          # same tolerance as the parity tests
         assert np.max(np.abs(new - want)) <= TOL * scale         # and right against the oracle, not merely equal
         assert np.array_equal(new, ref)                          # same arithmetic in the same order: identical bits
+
+
+def test_requantised_output_through_the_entry_point_that_allocates_nothing():
+    """The packed-codes output (the next site's quantiser in the epilogue) gives the same bytes through
+    both entry points."""
+    import torch
+    from paper_2304_01089_b200 import binding
+    rng = np.random.default_rng(31)
+    M, C, g, bits = 200, 512, 4, 4
+    perm2, size2, scale2, zero2 = random_layout_params(rng, 352, 3, 3, allow_empty=False)
+    L2 = binding.Layout(perm2, size2, (scale2 * 0.2).astype(np.float32), zero2, 3)
+    N = L2.K_pad
+    dev, _ = _problem(rng, M, N, C, g, bits)
+    outs = []
+    for fn in (binding.cluster_gemm, binding.cluster_gemm_noalloc, binding.cluster_gemm_noalloc):
+        y = torch.full((M + 1, L2.row_bytes), 0xA5, dtype=torch.uint8, device="cuda")
+        fn(dev["L"], dev["a"], M, dev["w"], dev["s_w"], dev["wsum"], N, y, bias=dev["bias"], act=binding.ACT_RELU,
+           layout_out=L2, y_dtype=binding.OUT_CODES)
+        torch.cuda.synchronize()
+        out = y.cpu().numpy()
+        assert np.all(out[M] == 0xA5)
+        outs.append(out[:M])
+    assert np.array_equal(outs[0], outs[1]) and np.array_equal(outs[1], outs[2])
+    codes = oracle.unpack(outs[1], N, 3)
+    assert codes.max() <= 7 and not codes[:, L2.padded_index() < 0].any() and codes.any()
 
 
 def test_more_columns_than_the_resident_table_is_refused():
