@@ -183,6 +183,43 @@ int rptq_cluster_gemm(const rptq_layout_t* Lin, const void* a_codes, int M, cons
                       void* stream);
 
 /*
+ * Appendix: "for one output channel, each weight cluster is quantised with its own asymmetric
+ * parameters", W~_q,i = Q_k(W~_i, s^W_i, z^W_i), the paper's own weight scheme (it finds the codes
+ * with GPTQ; here round-to-nearest). For output row r and input cluster c with n_c > 0, in fp32:
+ *   s = (max - min) / 16 over the row's weights of the cluster (1 if max == min)       [Eq. 2, k = 4]
+ *   z = 8 - rne((max + min) / (2 s)),   W_q = clamp(rne(W / s) + z, 0, 15)           [Eq. 1, re-based]
+ * The packed buffer has the format and size of rptq_weight_pack's; the stored nibble is W_q - 8.
+ *   s_w, z_w, wsum  host [g][N_pad]: scale, zero point of the codes in [0, 15], sum of the codes over
+ *                   the cluster's channels. Empty clusters and rows r >= N: s = 1, z = 0, sum 0.
+ */
+int rptq_weight_pack_clustered(const rptq_layout_t* Lin, const float* W_host, int N, int N_pad,
+                               void* w_codes_host, float* s_w, int32_t* z_w, int32_t* wsum);
+
+/*
+ * xsum[m][c] = sum of the activation codes of token m over the positions of cluster c (int32, dev
+ * [M][g]): the factor of z^W_c in the second computation method of the Appendix.
+ *   codes  dev, M rows of L.row_bytes bytes as written by rptq_ln_reorder_quant or an RPTQ_OUT_CODES GEMM
+ * g <= 8192.
+ */
+int rptq_code_rowsums(const rptq_layout_t* L, const void* codes, int M, int32_t* xsum, void* stream);
+
+/*
+ * Appendix, second computation method with all four terms (the printed expression leaves the sums
+ * and the cluster size out):
+ *   Y_q,c[m][n] = sum_k X_q W_q - z^X_c sum_k W_q - z^W_c[n] sum_k X_q + n_c z^X_c z^W_c[n]   (k over cluster c)
+ *   y[m][n]     = sum_c s^X_c s^W_c[n] Y_q,c[m][n]  (+ bias[n]) (ReLU), re-quantised if asked for
+ * with the integer products exact on the tensor cores and the rest in fp32. Arguments as for
+ * rptq_cluster_gemm, except:
+ *   xsum           dev int32 [M][g] from rptq_code_rowsums on a_codes
+ *   w_codes, s_w, z_w, wsum  as produced by rptq_weight_pack_clustered and copied to the device; the
+ *                  three tables are [g][ld_w] with ld_w = N_pad a multiple of 4
+ */
+int rptq_cluster_gemm_clustered(const rptq_layout_t* Lin, const void* a_codes, int M, const int32_t* xsum,
+                                const void* w_codes, const float* s_w, const int32_t* z_w, const int32_t* wsum,
+                                int64_t ld_w, const void* bias, int N, int act, const rptq_layout_t* Lout,
+                                void* y, int y_dtype, int64_t ldy, void* stream);
+
+/*
  * The same operation as rptq_cluster_gemm, arguments and results included, for callers that must
  * not allocate device memory. (The paper has no counterpart; this is a property of the library.)
  * Who needs it: a process whose device memory is owned wholesale by its own pool -- an inference

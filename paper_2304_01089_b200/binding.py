@@ -26,7 +26,7 @@ EXPORTS = (
     "rptq_weight_pack", "rptq_cluster_gemm", "rptq_cluster_gemm_debug_acc", "rptq_codes_unpack_host",
     "rptq_codes_pack_host", "rptq_weight_unpack_host", "rptq_get_device_status", "rptq_status_string",
     "rptq_format_version", "rptq_layout_padded_index", "rptq_weight_codes_bytes", "rptq_cluster_gemm_noalloc",
-    "rptq_probe_int8_peak",
+    "rptq_probe_int8_peak", "rptq_weight_pack_clustered", "rptq_code_rowsums", "rptq_cluster_gemm_clustered",
 )
 
 
@@ -56,6 +56,9 @@ def _load(path: str = LIB_PATH) -> C.CDLL:
     lib.rptq_codes_pack_host.argtypes = [i32, i32, vp, i64, vp]
     lib.rptq_weight_unpack_host.argtypes = [i32, vp, i64, vp]
     lib.rptq_weight_codes_bytes.argtypes = [i32, i64]
+    lib.rptq_weight_pack_clustered.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp]
+    lib.rptq_code_rowsums.argtypes = [vp, vp, i32, vp, vp]
+    lib.rptq_cluster_gemm_clustered.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp, i64, vp, i32, i32, vp, vp, i32, i64, vp]
     lib.rptq_probe_int8_peak.argtypes = [i32, vp, C.POINTER(C.c_double), vp]
     lib.rptq_get_device_status.argtypes = [C.POINTER(i32)]
     lib.rptq_status_string.argtypes = [i32]
@@ -220,6 +223,41 @@ def cluster_gemm(layout_in: Layout, a_codes, M: int, w_codes, s_w, wsum, N: int,
                                   _dev_ptr(wsum), ld_w, _dev_ptr(bias), int(N), int(act),
                                   None if layout_out is None else layout_out.handle, _dev_ptr(y), int(y_dtype),
                                   int(ldy), _stream_ptr(stream)), "rptq_cluster_gemm")
+
+
+def weight_pack_clustered(layout_in: Layout, W: np.ndarray, n_pad: Optional[int] = None):
+    """rptq_weight_pack_clustered on host arrays. Returns (w_codes flat uint8 tile-major buffer,
+    s_w fp32 [g][N_pad], z_w int32 [g][N_pad], wsum int32 [g][N_pad])."""
+    W = np.ascontiguousarray(W, dtype=np.float32)
+    N, Cn = W.shape
+    if Cn != layout_in.C:
+        raise ValueError("W must be [N][C] with C the layout's channel count")
+    n_pad = N if n_pad is None else int(n_pad)
+    w_codes = np.empty(weight_codes_bytes(layout_in.K_pad, n_pad), np.uint8)
+    s_w = np.empty((layout_in.g, n_pad), np.float32)
+    z_w = np.empty((layout_in.g, n_pad), np.int32)
+    wsum = np.empty((layout_in.g, n_pad), np.int32)
+    _check(_lib.rptq_weight_pack_clustered(layout_in.handle, _np_ptr(W), N, n_pad, _np_ptr(w_codes), _np_ptr(s_w),
+                                           _np_ptr(z_w), _np_ptr(wsum)), "rptq_weight_pack_clustered")
+    return w_codes, s_w, z_w, wsum
+
+
+def code_rowsums(layout: Layout, codes, M: int, xsum, stream=None) -> None:
+    """rptq_code_rowsums: xsum int32 [M][g] device tensor."""
+    _check(_lib.rptq_code_rowsums(layout.handle, _dev_ptr(codes), int(M), _dev_ptr(xsum), _stream_ptr(stream)), "rptq_code_rowsums")
+
+
+def cluster_gemm_clustered(layout_in: Layout, a_codes, M: int, xsum, w_codes, s_w, z_w, wsum, N: int, y, *,
+                           bias=None, act: int = ACT_NONE, layout_out: Optional[Layout] = None, y_dtype: int = OUT_F32,
+                           ldy: Optional[int] = None, stream=None) -> None:
+    """rptq_cluster_gemm_clustered on device tensors (s_w, z_w, wsum are [g][N_pad])."""
+    ld_w = int(s_w.shape[1])
+    if ldy is None:
+        ldy = 0 if y_dtype == OUT_CODES else int(y.stride(0))
+    _check(_lib.rptq_cluster_gemm_clustered(layout_in.handle, _dev_ptr(a_codes), int(M), _dev_ptr(xsum), _dev_ptr(w_codes),
+                                            _dev_ptr(s_w), _dev_ptr(z_w), _dev_ptr(wsum), ld_w, _dev_ptr(bias), int(N), int(act),
+                                            None if layout_out is None else layout_out.handle, _dev_ptr(y), int(y_dtype),
+                                            int(ldy), _stream_ptr(stream)), "rptq_cluster_gemm_clustered")
 
 
 def cluster_gemm_noalloc(layout_in: Layout, a_codes, M: int, w_codes, s_w, wsum, N: int, y, *, ld_w: Optional[int] = None,

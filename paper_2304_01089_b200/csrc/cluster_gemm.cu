@@ -100,6 +100,13 @@ struct Params {
     const float* s_w;
     const int32_t* wsum;
     int64_t ld_w;
+    // per-cluster asymmetric weight parameters (template flag ASYM): [g][ld_w] tables of s^W_c[n] and
+    // z^W_c[n], the cluster of every entry of seg_scale, n_c, and the activation code sums [M][g]
+    const float* sw_c;
+    const int32_t* zw_c;
+    const int32_t* seg_cluster;
+    const float* cl_n;
+    const int32_t* xsum;
     const float* bias;
     int act, y_dtype;
     void* y;
@@ -299,7 +306,13 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr)
     return v;
 }
 
-template <int BITS, int NCTA, bool A8>
+// ASYM: the weights carry one scale and one zero point per (cluster, output channel) (Appendix,
+// W~_q,i = Q_k(W~_i, s^W_i, z^W_i)). The stored nibble is the code minus 8, so the integer products
+// are acc' = sum X_q (W_q - 8) and the second method's four terms become
+//   Y_q,c = acc'_c - (z^W_c[n] - 8) * sum_k X_q[m][k] - z^X_c * Wsum_c[n] + n_c z^X_c z^W_c[n] :
+// the first two are applied per element while a cluster's accumulator is drained, the last two are a
+// constant of the output column.
+template <int BITS, int NCTA, bool A8, bool ASYM>
 __global__ void __launch_bounds__(THREADS, 1)
 cluster_gemm_kernel(const Params p)
 {
@@ -655,9 +668,19 @@ cluster_gemm_kernel(const Params p)
                 const int n = n0 + et;
                 float corr = 0.f, sw = 0.f, bs = 0.f;
                 if (n < p.N) {
-                    if (p.corr) corr = __ldg(p.corr + n);
-                    else for (int c = 0; c < p.g; ++c) corr = __fmaf_rn(s_cl_sz[c], (float)__ldg(p.wsum + (int64_t)c * p.ld_w + n), corr);
-                    sw = __ldg(p.s_w + n);
+                    if constexpr (ASYM) {
+                        // sum_c s^X_c z^X_c s^W_c[n] (Wsum_c[n] - n_c z^W_c[n]); the column's scale is applied per cluster
+                        for (int c = 0; c < p.g; ++c) {
+                            const int64_t i = (int64_t)c * p.ld_w + n;
+                            const float t = (float)__ldg(p.wsum + i) - __ldg(p.cl_n + c) * (float)__ldg(p.zw_c + i);
+                            corr = __fmaf_rn(s_cl_sz[c] * __ldg(p.sw_c + i), t, corr);
+                        }
+                        sw = 1.0f;
+                    } else {
+                        if (p.corr) corr = __ldg(p.corr + n);
+                        else for (int c = 0; c < p.g; ++c) corr = __fmaf_rn(s_cl_sz[c], (float)__ldg(p.wsum + (int64_t)c * p.ld_w + n), corr);
+                        sw = __ldg(p.s_w + n);
+                    }
                     bs = p.bias ? __ldg(p.bias + n) : 0.f;
                 }
                 tab[et] = corr; tab[TILE_N + et] = sw; tab[2 * TILE_N + et] = bs;
@@ -676,11 +699,44 @@ cluster_gemm_kernel(const Params p)
                 const uint32_t taddr = tmem_base + ((uint32_t)(32 * q) << 16) + buf * TILE_N + h * 128;
                 uint32_t va[16], vb[16];
                 tc_ld16(taddr, va);
+                // ASYM: this cluster's row of the weight tables and my token's code sum
+                int64_t tab_row = 0;
+                float xs = 0.f, sx = 0.f;
+                if constexpr (ASYM) {
+                    const int cid = __ldg(p.seg_cluster + sgi);
+                    const int m_row = m0 + 32 * q + lane;
+                    tab_row = (int64_t)cid * p.ld_w + n0 + h * 128;
+                    xs = m_row < p.M ? (float)__ldg(p.xsum + (int64_t)m_row * p.g + cid) : 0.f;
+                    sx = sc * 16.0f;                 // s^X_c itself (s_seg_scale carries the 1/16 of the operands)
+                }
                 // R += s_c * acc, two columns per packed fused multiply-add
                 auto accumulate = [&](const uint32_t (&v)[16], int c0) {
+                    if constexpr (ASYM) {
+                        // R += s^X_c s^W_c[n] (acc' - (z^W_c[n] - 8) xsum): 16 columns, the tables four at a time
+                        const int col = 2 * c0;                      // first of these columns within my 128
 #pragma unroll
-                    for (int i = 0; i < 8; ++i)
-                        R[c0 + i] = fma2(sc2, make_float2((float)(int)v[2 * i], (float)(int)v[2 * i + 1]), R[c0 + i]);
+                        for (int i4 = 0; i4 < 4; ++i4) {
+                            float sw4[4] = {0.f, 0.f, 0.f, 0.f};
+                            int zw4[4] = {8, 8, 8, 8};
+                            if (n0 + h * 128 + col + 4 * i4 + 4 <= p.ld_w) {
+                                const float4 a = __ldg(reinterpret_cast<const float4*>(p.sw_c + tab_row + col + 4 * i4));
+                                const int4 b = __ldg(reinterpret_cast<const int4*>(p.zw_c + tab_row + col + 4 * i4));
+                                sw4[0] = a.x; sw4[1] = a.y; sw4[2] = a.z; sw4[3] = a.w;
+                                zw4[0] = b.x; zw4[1] = b.y; zw4[2] = b.z; zw4[3] = b.w;
+                            }
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const int i = 4 * i4 + e;
+                                const float t = __fmaf_rn((float)(int)v[i], 0.0625f, -(float)(zw4[e] - 8) * xs);
+                                float& r = (i & 1) ? R[c0 + (i >> 1)].y : R[c0 + (i >> 1)].x;
+                                r = __fmaf_rn(sx * sw4[e], t, r);
+                            }
+                        }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            R[c0 + i] = fma2(sc2, make_float2((float)(int)v[2 * i], (float)(int)v[2 * i + 1]), R[c0 + i]);
+                    }
                 };
 #pragma unroll
                 for (int ch = 0; ch < 8; ch += 2) {
@@ -781,12 +837,12 @@ cluster_gemm_kernel(const Params p)
 }
 
 // ---------------------------------------------------------------- host side
-template <int BITS, int NCTA, bool A8>
+template <int BITS, int NCTA, bool A8, bool ASYM>
 static int launch(const Params& p, int n_sm, cudaStream_t st)
 {
     constexpr SmemLayout SL = smem_layout(NCTA, BITS, A8);
     const int smem = SL.total + 1024;     // slack for the in-kernel 1024-byte alignment
-    const void* fn = reinterpret_cast<const void*>(cluster_gemm_kernel<BITS, NCTA, A8>);
+    const void* fn = reinterpret_cast<const void*>(cluster_gemm_kernel<BITS, NCTA, A8, ASYM>);
     cudaFuncAttributes attr;
     if (cudaFuncGetAttributes(&attr, fn) != cudaSuccess) return RPTQ_ERR_CUDA;
     // the register re-partition inside the kernel (setmaxnreg) assumes this pool; refuse to launch otherwise
@@ -804,7 +860,7 @@ static int launch(const Params& p, int n_sm, cudaStream_t st)
     at[0].val.clusterDim.x = NCTA; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
     cfg.attrs = at;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, cluster_gemm_kernel<BITS, NCTA, A8>, p) == cudaSuccess ? RPTQ_OK : RPTQ_ERR_CUDA;
+    return cudaLaunchKernelEx(&cfg, cluster_gemm_kernel<BITS, NCTA, A8, ASYM>, p) == cudaSuccess ? RPTQ_OK : RPTQ_ERR_CUDA;
 }
 
 }  // namespace gemm
@@ -843,7 +899,8 @@ static int check_gemm_args(const rptq_layout_t* Lin, const void* a_codes, int M,
 static int launch_gemm(const rptq_layout_t* Lin, const void* a_codes, int M, const void* w_codes,
                        const float* s_w, const int32_t* wsum, int64_t ld_w, const void* bias, int N,
                        int act, const rptq_layout_t* Lout, void* y, int y_dtype, int64_t ldy, void* stream,
-                       int dev, int* status, const float* corr)
+                       int dev, int* status, const float* corr,
+                       const float* sw_c = nullptr, const int32_t* zw_c = nullptr, const int32_t* xsum = nullptr)
 {
     gemm::Params p{};
     p.M = M; p.N = N; p.n_kb = Lin->K_pad / gemm::KBLK; p.n_seg = Lin->n_seg; p.g = Lin->g;
@@ -861,18 +918,46 @@ static int launch_gemm(const rptq_layout_t* Lin, const void* a_codes, int M, con
     p.out_row_bytes = Lout ? Lout->row_bytes : 0;
     p.status = status;
     p.corr = corr;
+    p.sw_c = sw_c; p.zw_c = zw_c; p.xsum = xsum; p.seg_cluster = Lin->d_seg_cluster; p.cl_n = Lin->d_cl_n;
 
     int n_sm = 0;
     if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return RPTQ_ERR_CUDA;
     auto st = static_cast<cudaStream_t>(stream);
-    if (ncta == 2) {
-        if (Lin->bits == 3) return gemm::launch<3, 2, false>(p, n_sm, st);
-        if (Lin->bits == 4) return gemm::launch<4, 2, false>(p, n_sm, st);
-        return gemm::launch<8, 2, true>(p, n_sm, st);      // 8-bit codes need no unpacking
+    if (sw_c) {
+        if (ncta == 2) {
+            if (Lin->bits == 3) return gemm::launch<3, 2, false, true>(p, n_sm, st);
+            if (Lin->bits == 4) return gemm::launch<4, 2, false, true>(p, n_sm, st);
+            return gemm::launch<8, 2, true, true>(p, n_sm, st);
+        }
+        if (Lin->bits == 3) return gemm::launch<3, 1, false, true>(p, n_sm, st);
+        if (Lin->bits == 4) return gemm::launch<4, 1, false, true>(p, n_sm, st);
+        return gemm::launch<8, 1, false, true>(p, n_sm, st);
     }
-    if (Lin->bits == 3) return gemm::launch<3, 1, false>(p, n_sm, st);
-    if (Lin->bits == 4) return gemm::launch<4, 1, false>(p, n_sm, st);
-    return gemm::launch<8, 1, false>(p, n_sm, st);
+    if (ncta == 2) {
+        if (Lin->bits == 3) return gemm::launch<3, 2, false, false>(p, n_sm, st);
+        if (Lin->bits == 4) return gemm::launch<4, 2, false, false>(p, n_sm, st);
+        return gemm::launch<8, 2, true, false>(p, n_sm, st);      // 8-bit codes need no unpacking
+    }
+    if (Lin->bits == 3) return gemm::launch<3, 1, false, false>(p, n_sm, st);
+    if (Lin->bits == 4) return gemm::launch<4, 1, false, false>(p, n_sm, st);
+    return gemm::launch<8, 1, false, false>(p, n_sm, st);
+}
+
+extern "C" int rptq_cluster_gemm_clustered(const rptq_layout_t* Lin, const void* a_codes, int M, const int32_t* xsum,
+                                           const void* w_codes, const float* s_w, const int32_t* z_w, const int32_t* wsum,
+                                           int64_t ld_w, const void* bias, int N, int act, const rptq_layout_t* Lout,
+                                           void* y, int y_dtype, int64_t ldy, void* stream)
+{
+    int dev = -1;
+    const int rc = check_gemm_args(Lin, a_codes, M, w_codes, s_w, wsum, ld_w, bias, N, act, Lout, y, y_dtype, ldy, &dev);
+    if (rc != RPTQ_OK) return rc;
+    if (!z_w || !xsum || !aligned16(z_w) || !aligned16(xsum)) return RPTQ_ERR_INVALID_ARG;
+    if (ld_w % 4 != 0) return RPTQ_ERR_UNSUPPORTED;       // the tables are read four columns at a time
+    if (M == 0) return RPTQ_OK;
+    int* status = device_status_word();
+    if (!status) return RPTQ_ERR_ALLOC;
+    return launch_gemm(Lin, a_codes, M, w_codes, nullptr, wsum, ld_w, bias, N, act, Lout, y, y_dtype, ldy, stream, dev, status,
+                       nullptr, s_w, z_w, xsum);
 }
 
 extern "C" int rptq_cluster_gemm(const rptq_layout_t* Lin, const void* a_codes, int M, const void* w_codes,

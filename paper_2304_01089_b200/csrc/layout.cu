@@ -210,12 +210,13 @@ int rptq_layout_create(rptq_layout_t** out, int C, int g, int bits, const int32_
     std::vector<int32_t> jidx((size_t)k_pad, -1);                // reordered index at each position, -1 at pads
     std::vector<UnitInfo> unit((size_t)L->n_units);
     std::vector<uint8_t> flags((size_t)L->n_units, STEP_SKIP);
-    std::vector<float> seg_scale, cl_sz((size_t)g);
+    std::vector<float> seg_scale, cl_sz((size_t)g), cl_n((size_t)g);
+    std::vector<int32_t> seg_cluster;
     std::vector<uint8_t> seg_buf;
     L->unit_cluster.assign((size_t)L->n_units, -1);
     L->pos.assign((size_t)C, 0);
     for (auto& u : unit) { u.inv_s = 1.0f; u.zc = 0 - 0x4B400000; u.j0 = 0; u.nvalid = 0; }
-    for (int c = 0; c < g; ++c) cl_sz[c] = scale_host[c] * (float)zero_host[c];
+    for (int c = 0; c < g; ++c) { cl_sz[c] = scale_host[c] * (float)zero_host[c]; cl_n[c] = (float)cluster_size[c]; }
     // Accumulator of each cluster: the one that is not held by a cluster still under way; when
     // both are free, the one whose last cluster ended longer ago (its drain has had more time).
     int last_end[2] = {-2, -1};              // unit index at which each accumulator's last cluster ended
@@ -238,6 +239,7 @@ int rptq_layout_create(rptq_layout_t** out, int C, int g, int bits, const int32_
                 last_end[buf_of[c]] = cur;
                 seg_scale.push_back(scale_host[c]);
                 seg_buf.push_back((uint8_t)buf_of[c]);
+                seg_cluster.push_back(c);
                 L->n_seg++;
                 if (open_cluster == c) { open_cluster = -1; open_buf = -1; }
             }
@@ -303,6 +305,8 @@ int rptq_layout_create(rptq_layout_t** out, int C, int g, int bits, const int32_
     if (rc == RPTQ_OK) rc = upload(&L->d_seg_scale, seg_scale.data(), seg_scale.size());
     if (rc == RPTQ_OK) rc = upload(&L->d_cl_sz, cl_sz.data(), cl_sz.size());
     if (rc == RPTQ_OK) rc = upload(&L->d_seg_buf, seg_buf.data(), seg_buf.size());
+    if (rc == RPTQ_OK) rc = upload(&L->d_cl_n, cl_n.data(), cl_n.size());
+    if (rc == RPTQ_OK) rc = upload(&L->d_seg_cluster, seg_cluster.data(), seg_cluster.size());
     if (rc == RPTQ_OK) rc = upload(&L->d_unit_cluster, L->unit_cluster.data(), L->unit_cluster.size());
     if (rc != RPTQ_OK) { rptq_layout_destroy(L); return rc; }
     *out = L;
@@ -336,6 +340,8 @@ int rptq_layout_destroy(rptq_layout_t* L)
     cudaFree(L->d_seg_scale);
     cudaFree(L->d_cl_sz);
     cudaFree(L->d_seg_buf);
+    cudaFree(L->d_cl_n);
+    cudaFree(L->d_seg_cluster);
     cudaFree(L->d_unit_cluster);
     delete L;
     return RPTQ_OK;
@@ -433,6 +439,68 @@ int rptq_weight_pack(const rptq_layout_t* Lin, const float* W_host, int N, const
                 for (int c = 0; c < g; ++c) wsum[(int64_t)c * N_pad + r] = 0;
             }
             s_w[r] = s;
+            pack_row(row.data(), K_pad, 4, row_packed.data());
+            for (int kb = 0; kb < n_kb; ++kb) std::memcpy(packed + weight_tile_offset(r, kb, n_kb), row_packed.data() + 64 * kb, 64);
+        }
+    }
+    return failed ? RPTQ_ERR_INVALID_ARG : RPTQ_OK;
+}
+
+int rptq_weight_pack_clustered(const rptq_layout_t* Lin, const float* W_host, int N, int N_pad,
+                               void* w_codes_host, float* s_w, int32_t* z_w, int32_t* wsum)
+{
+    if (!Lin || !W_host || !w_codes_host || !s_w || !z_w || !wsum) return RPTQ_ERR_INVALID_ARG;
+    if (N <= 0 || N_pad < N) return RPTQ_ERR_INVALID_ARG;
+    const int C = Lin->C, g = Lin->g, K_pad = Lin->K_pad;
+    const int n_kb = K_pad / 128;
+    const int rows_stored = (N_pad + 127) / 128 * 128;
+    uint8_t* packed = static_cast<uint8_t*>(w_codes_host);
+    std::vector<int> j_start((size_t)g);
+    for (int c = 0, j = 0; c < g; ++c) { j_start[c] = j; j += Lin->size[c]; }
+    int failed = 0;
+#pragma omp parallel
+    {
+        std::vector<uint8_t> row((size_t)K_pad), row_packed((size_t)K_pad / 2);
+#pragma omp for schedule(static)
+        for (int r = 0; r < rows_stored; ++r) {
+            if (r >= N_pad) {
+                for (int kb = 0; kb < n_kb; ++kb) std::memset(packed + weight_tile_offset(r, kb, n_kb), 0, 64);
+                continue;
+            }
+            // positions that hold no channel, and rows past N, store code 8 (the nibble 0)
+            std::memset(row.data(), 0, (size_t)K_pad);
+            for (int c = 0; c < g; ++c) {
+                float s = 1.0f;
+                int32_t z = 0, sum = 0;
+                const int n_c = Lin->size[c];
+                if (r < N && n_c > 0) {
+                    const float* w = W_host + (int64_t)r * C;
+                    float lo = INFINITY, hi = -INFINITY;
+                    for (int i = 0; i < n_c; ++i) {
+                        const float v = w[Lin->perm[j_start[c] + i]];
+                        lo = fminf(lo, v); hi = fmaxf(hi, v);
+                    }
+                    if (!std::isfinite(lo) || !std::isfinite(hi)) {
+#pragma omp atomic write
+                        failed = 1;
+                    }
+                    s = (hi - lo) / 16.0f;                              // Eq. 2, k = 4
+                    if (!(s > 0.0f)) s = 1.0f;
+                    const float mid = (hi + lo) / (2.0f * s);
+                    z = 8 - (int32_t)rintf(mid);
+                    for (int i = 0; i < n_c; ++i) {
+                        const int j = j_start[c] + i;
+                        float q = rintf(w[Lin->perm[j]] / s) + (float)z;   // Eq. 1
+                        q = fminf(fmaxf(q, 0.0f), 15.0f);
+                        const int qi = (int)q;
+                        sum += qi;
+                        row[Lin->pos[j]] = (uint8_t)((qi - 8) & 0xF);
+                    }
+                }
+                s_w[(int64_t)c * N_pad + r] = s;
+                z_w[(int64_t)c * N_pad + r] = z;
+                wsum[(int64_t)c * N_pad + r] = sum;
+            }
             pack_row(row.data(), K_pad, 4, row_packed.data());
             for (int kb = 0; kb < n_kb; ++kb) std::memcpy(packed + weight_tile_offset(r, kb, n_kb), row_packed.data() + 64 * kb, 64);
         }

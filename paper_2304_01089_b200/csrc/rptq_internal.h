@@ -48,6 +48,8 @@ struct rptq_layout {
     float* d_seg_scale = nullptr;       // [n_seg]  s_c of the non-empty clusters, in the order their last steps come
     uint8_t* d_seg_buf = nullptr;       // [n_seg]  the accumulator each of them uses, same order
     float* d_cl_sz = nullptr;           // [g]      s_c * z_c
+    float* d_cl_n = nullptr;            // [g]      n_c
+    int32_t* d_seg_cluster = nullptr;   // [n_seg]  the cluster of each entry of d_seg_scale
     int32_t* d_unit_cluster = nullptr;  // [n_units]
 };
 
