@@ -272,6 +272,35 @@ int64_t rptq_weight_codes_bytes(int K_pad, int64_t N_pad);
 int rptq_get_device_status(int* status);
 
 /*
+ * Calibration on the device (Sec. 4.1), off the hot path.
+ *
+ * Eq. 3 at a LayerNorm site: x_min[c], x_max[c] = minimum and maximum of the LayerNorm output of
+ * channel c over T calibration tokens (LayerNorm in fp32 with the arithmetic of
+ * rptq_ln_reorder_quant). x dev fp16 [T][ldx], gamma / beta dev fp16 [C], x_min / x_max dev fp32 [C]
+ * (overwritten). C <= 16384.
+ */
+int rptq_ln_channel_minmax(const void* x, int64_t ldx, const void* gamma, const void* beta, float eps,
+                           int T, int C, float* x_min, float* x_max, void* stream);
+
+/*
+ * Sec. 4.1: K-Means of n points (the channels' (min, max) pairs: dim = 2; Sec. 4.2 clusters Q and K
+ * together on (Q_max, Q_min, K_max, K_min): dim = 4) into g clusters. The paper names the algorithm
+ * only; the steps are: k-means++ seeding driven by the uniform draws u[0..g-1] (u[0] picks the first
+ * centre, u[k] the point at which the running sum of squared distances to the nearest chosen centre
+ * passes u[k] times its total), then `iters` Lloyd iterations with squared Euclidean distance in fp64,
+ * ties to the lowest centre, a centre without points re-seeded at the point farthest from its own
+ * centre. All sums run in point order, so a sequential program taking the same steps gives the same
+ * labels.
+ *   pts dev fp64 [n][dim], u dev fp64 [g], labels dev int32 [n], centres dev fp64 [g][dim],
+ *   inertia NULL or dev fp64 [iters] (sum of squared distances at each assignment step),
+ *   workspace dev, rptq_kmeans_workspace_bytes(n, g) bytes, 8-byte aligned. dim <= 8.
+ * One thread block does all of it: seconds for tens of thousands of points and hundreds of clusters.
+ */
+int64_t rptq_kmeans_workspace_bytes(int n, int g);
+int rptq_kmeans(const double* pts, int n, int dim, int g, const double* u, int iters, int32_t* labels,
+                double* centres, double* inertia, void* workspace, void* stream);
+
+/*
  * Measurement aid (the paper has no counterpart): launches, on `stream`, a kernel that issues the
  * cluster GEMM's own tensor-core instruction -- tcgen05.mma kind::i8 over CTA pairs, 256 x 256 x 32,
  * unsigned x signed 8-bit into int32 -- back to back on operands resident in shared memory, with no

@@ -26,6 +26,7 @@ EXPORTS = (
     "rptq_weight_pack", "rptq_cluster_gemm", "rptq_cluster_gemm_debug_acc", "rptq_codes_unpack_host",
     "rptq_codes_pack_host", "rptq_weight_unpack_host", "rptq_get_device_status", "rptq_status_string",
     "rptq_format_version", "rptq_layout_padded_index", "rptq_weight_codes_bytes", "rptq_cluster_gemm_noalloc",
+    "rptq_ln_channel_minmax", "rptq_kmeans", "rptq_kmeans_workspace_bytes",
     "rptq_probe_int8_peak", "rptq_weight_pack_clustered", "rptq_code_rowsums", "rptq_cluster_gemm_clustered",
 )
 
@@ -56,6 +57,9 @@ def _load(path: str = LIB_PATH) -> C.CDLL:
     lib.rptq_codes_pack_host.argtypes = [i32, i32, vp, i64, vp]
     lib.rptq_weight_unpack_host.argtypes = [i32, vp, i64, vp]
     lib.rptq_weight_codes_bytes.argtypes = [i32, i64]
+    lib.rptq_ln_channel_minmax.argtypes = [vp, i64, vp, vp, f32, i32, i32, vp, vp, vp]
+    lib.rptq_kmeans_workspace_bytes.argtypes = [i32, i32]
+    lib.rptq_kmeans.argtypes = [vp, i32, i32, i32, vp, i32, vp, vp, vp, vp, vp]
     lib.rptq_weight_pack_clustered.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp]
     lib.rptq_code_rowsums.argtypes = [vp, vp, i32, vp, vp]
     lib.rptq_cluster_gemm_clustered.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp, i64, vp, i32, i32, vp, vp, i32, i64, vp]
@@ -64,9 +68,10 @@ def _load(path: str = LIB_PATH) -> C.CDLL:
     lib.rptq_status_string.argtypes = [i32]
     lib.rptq_status_string.restype = C.c_char_p
     for name in EXPORTS:
-        if name not in ("rptq_status_string", "rptq_weight_codes_bytes"):
+        if name not in ("rptq_status_string", "rptq_weight_codes_bytes", "rptq_kmeans_workspace_bytes"):
             getattr(lib, name).restype = i32
     lib.rptq_weight_codes_bytes.restype = i64
+    lib.rptq_kmeans_workspace_bytes.restype = i64
     return lib
 
 
@@ -310,6 +315,26 @@ def weight_unpack_host(packed: np.ndarray, k_pad: int, n_rows: int) -> np.ndarra
     out = np.empty((N, k_pad), np.int8)
     _check(_lib.rptq_weight_unpack_host(int(k_pad), _np_ptr(packed), N, _np_ptr(out)), "rptq_weight_unpack_host")
     return out
+
+
+def ln_channel_minmax(x, gamma, beta, eps: float, x_min, x_max, T: Optional[int] = None, stream=None) -> None:
+    """rptq_ln_channel_minmax: x fp16 [T][ldx], gamma / beta fp16 [C], x_min / x_max fp32 [C] device tensors."""
+    T = int(x.shape[0]) if T is None else int(T)
+    _check(_lib.rptq_ln_channel_minmax(_dev_ptr(x), int(x.stride(0)), _dev_ptr(gamma), _dev_ptr(beta), C.c_float(eps), T,
+                                       int(gamma.shape[0]), _dev_ptr(x_min), _dev_ptr(x_max), _stream_ptr(stream)),
+           "rptq_ln_channel_minmax")
+
+
+def kmeans(pts, g: int, u, iters: int, labels, centres, inertia, workspace, stream=None) -> None:
+    """rptq_kmeans on device tensors: pts fp64 [n][dim], u fp64 [g], labels int32 [n], centres fp64 [g][dim],
+    inertia fp64 [iters] or None, workspace uint8 of kmeans_workspace_bytes(n, g) bytes."""
+    n, dim = int(pts.shape[0]), int(pts.shape[1])
+    _check(_lib.rptq_kmeans(_dev_ptr(pts), n, dim, int(g), _dev_ptr(u), int(iters), _dev_ptr(labels), _dev_ptr(centres),
+                            _dev_ptr(inertia), _dev_ptr(workspace), _stream_ptr(stream)), "rptq_kmeans")
+
+
+def kmeans_workspace_bytes(n: int, g: int) -> int:
+    return int(_lib.rptq_kmeans_workspace_bytes(int(n), int(g)))
 
 
 def probe_int8_peak(n_batches: int, failed, stream=None) -> float:

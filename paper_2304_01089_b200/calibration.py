@@ -128,10 +128,12 @@ def reorder_index(labels: np.ndarray, x_min: np.ndarray, x_max: np.ndarray, g: i
     return perm, size, new_of_old
 
 
-def calibrate_from_minmax(x_min, x_max, g: int, k: int, draws, iters: int = 20) -> Calibration:
+def calibrate_from_minmax(x_min, x_max, g: int, k: int, draws, iters: int = 20, labels=None) -> Calibration:
+    """`labels`: the clustering of the channels when it was computed elsewhere (on the device)."""
     x_min, x_max = np.asarray(x_min, np.float64), np.asarray(x_max, np.float64)
-    labels, _, _ = kmeans(np.stack([x_min, x_max], axis=1), g, draws, iters)
-    perm, size, _ = reorder_index(labels, x_min, x_max, g)
+    if labels is None:
+        labels, _, _ = kmeans(np.stack([x_min, x_max], axis=1), g, draws, iters)
+    perm, size, _ = reorder_index(np.asarray(labels), x_min, x_max, g)
     scale, zero = np.ones(g, np.float32), np.full(g, 1 << (k - 1), np.int32)
     pos = 0
     for c in range(g):
@@ -149,6 +151,26 @@ def calibrate(x_cal16, gamma16, beta16, g: int, k: int, draws, eps: float = 1e-5
     y = layernorm_fp64(x_cal16, gamma16, beta16, eps)
     x_min, x_max = channel_minmax(y)
     return calibrate_from_minmax(x_min, x_max, g, k, draws, iters)
+
+
+def calibrate_on_device(x_cal, gamma, beta, g: int, k: int, draws, eps: float = 1e-5, iters: int = 20) -> Calibration:
+    """The same calibration with the two heavy steps on the GPU (Sec. 4.1): the per-channel ranges of
+    Eq. 3 over the calibration tokens (rptq_ln_channel_minmax) and the K-Means of the channels
+    (rptq_kmeans). x_cal fp16 [T][C], gamma / beta fp16 [C]: CUDA tensors. The reorder index and the
+    per-cluster parameters of Eq. 2 are a few thousand operations and stay on the host."""
+    import torch
+    from . import binding
+    Cn = int(gamma.shape[0])
+    x_min = torch.empty(Cn, dtype=torch.float32, device=x_cal.device)
+    x_max = torch.empty_like(x_min)
+    binding.ln_channel_minmax(x_cal, gamma, beta, eps, x_min, x_max)
+    pts = torch.stack([x_min, x_max], dim=1).to(torch.float64).contiguous()
+    u = torch.from_numpy(np.ascontiguousarray(draws, dtype=np.float64)).to(x_cal.device)
+    labels = torch.empty(Cn, dtype=torch.int32, device=x_cal.device)
+    centres = torch.empty((g, 2), dtype=torch.float64, device=x_cal.device)
+    work = torch.empty(binding.kmeans_workspace_bytes(Cn, g), dtype=torch.uint8, device=x_cal.device)
+    binding.kmeans(pts, g, u, iters, labels, centres, None, work)
+    return calibrate_from_minmax(x_min.cpu().numpy(), x_max.cpu().numpy(), g, k, draws, iters, labels=labels.cpu().numpy())
 
 
 def segment_offsets(size: np.ndarray):
