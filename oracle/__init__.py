@@ -246,6 +246,21 @@ def dequant_matmul(a_codes, w_codes, size, scale, zero, s_w) -> np.ndarray:
     return y
 
 
+def dequant_matmul_bf16(a_codes, w_codes, size, scale32, zero, s_w, bias=None, relu=False) -> np.ndarray:
+    """First method with the de-quantised activation rounded to bfloat16 (the operand precision of a
+    16-bit tensor-core product)."""
+    a_codes, w_codes = _arr(a_codes, np.uint8), _arr(w_codes, np.int8)
+    size, zero = _arr(size, np.int32), _arr(zero, np.int32)
+    scale32, s_w = _arr(scale32, np.float32), _arr(s_w, np.float32)
+    M, k_pad = a_codes.shape
+    N = w_codes.shape[0]
+    b = None if bias is None else _arr(bias, np.float32)
+    y = np.empty((M, N))
+    _lib.orc_dequant_matmul_bf16(_p(a_codes), _i64(M), _p(w_codes), _i64(N), _i32(k_pad), C.c_int(size.shape[0]), _p(size),
+                                 _p(scale32), _p(zero), _p(s_w), _p(b), C.c_int(1 if relu else 0), _p(y))
+    return y
+
+
 # ---------------------------------------------------------------- per-cluster asymmetric weights
 def weight_quantize_clustered(W: np.ndarray, perm, size, k: int = 4, n_pad: Optional[int] = None):
     """Returns (w_codes uint8 [N_pad][K_pad], s_w fp32 [g][N_pad], z_w int32 [g][N_pad], wsum int32 [g][N_pad])."""

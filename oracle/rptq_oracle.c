@@ -700,3 +700,46 @@ void orc_dequant_matmul_asym(const uint8_t* a_codes, int64_t M, const uint8_t* w
         }
     free(seg_off);
 }
+
+/* ------------------------------------------------------------------------------------------ */
+/* First method with de-quantised operands of limited precision                                */
+/* ------------------------------------------------------------------------------------------ */
+
+/* round-to-nearest-even of an fp32 value to the bfloat16 format (8 bits of significand) */
+static float bf16_rne(float v)
+{
+    uint32_t u;
+    memcpy(&u, &v, 4);
+    if ((u & 0x7F800000u) != 0x7F800000u) u += 0x7FFFu + ((u >> 16) & 1u);
+    u &= 0xFFFF0000u;
+    memcpy(&v, &u, 4);
+    return v;
+}
+
+/* Appendix, first method, as a 16-bit floating-point matrix product computes it: the de-quantised
+ * activation X^ = s_c (X_q - z_c) is formed in fp32 (one multiply of the fp32 scale with the exact
+ * integer difference) and rounded to bfloat16; the weight operand is the integer code W_q, which
+ * bfloat16 holds exactly, and its scale s_w[n] multiplies the finished sum (W^ = s_w W_q, so that
+ * X^ W^ = s_w sum X^ W_q). The sum itself is exact here. Optional bias and ReLU as elsewhere. */
+void orc_dequant_matmul_bf16(const uint8_t* a_codes, int64_t M, const int8_t* w_codes, int64_t N,
+                             int32_t K_pad, int g, const int32_t* size, const float* scale32,
+                             const int32_t* zero, const float* s_w, const float* bias, int relu, double* y)
+{
+    int32_t* seg_off = (int32_t*)malloc(sizeof(int32_t) * (g + 1));
+    orc_segment_offsets(size, g, seg_off);
+#pragma omp parallel for schedule(static)
+    for (int64_t m = 0; m < M; ++m)
+        for (int64_t n = 0; n < N; ++n) {
+            double s = 0.0;
+            for (int c = 0; c < g; ++c)
+                for (int p = seg_off[c]; p < seg_off[c] + size[c]; ++p) {
+                    volatile float xh = scale32[c] * (float)((int32_t)a_codes[m * K_pad + p] - zero[c]);
+                    s += (double)bf16_rne(xh) * (double)w_codes[n * K_pad + p];
+                }
+            double v = (double)s_w[n] * s;
+            if (bias) v += (double)bias[n];
+            if (relu && v < 0.0) v = 0.0;
+            y[m * N + n] = v;
+        }
+    free(seg_off);
+}

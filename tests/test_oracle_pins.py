@@ -548,3 +548,45 @@ def test_code_rowsums_brute_force():
     for m in range(9):
         for ci, (o, n_c) in enumerate(zip(c["off"], c["size"])):
             assert got[m, ci] == sum(int(v) for v in c["a"][m, o:o + n_c])
+
+
+# ------------------------------------------------------------------ first method with bfloat16 operands
+def _bf16_round(v32):
+    """An independent statement of round-to-nearest-even to bfloat16: the nearer of the two
+    neighbouring 8-bit-significand values, the even one on a tie (by exact comparison in fp64)."""
+    u = np.asarray(v32, np.float32).view(np.uint32)
+    lo = (u & 0xFFFF0000).view(np.float32).astype(np.float64)             # truncation toward zero
+    hi = ((u & 0xFFFF0000) + np.uint32(0x10000)).view(np.float32).astype(np.float64)
+    x = np.asarray(v32, np.float64)
+    dl, dh = np.abs(x - lo), np.abs(hi - x)
+    even_lo = ((u >> 16) & 1) == 0
+    return np.where((dl < dh) | ((dl == dh) & even_lo), lo, hi)
+
+
+def test_bf16_first_method_against_numpy_and_within_its_rounding_bound():
+    r = _rng(41)
+    C, N, M, g = 160, 9, 7, 4
+    perm = r.permutation(C).astype(np.int32)
+    size = np.array([50, 3, 0, 107], np.int32)
+    W = (r.normal(size=(N, C)) * 0.02).astype(np.float32)
+    w, s_w, wsum = oracle.weight_quantize(W, perm, size)
+    off, k_pad = oracle.segment_offsets(size)
+    a = np.zeros((M, k_pad), np.uint8)
+    for c in range(g):
+        a[:, off[c]:off[c] + size[c]] = r.integers(0, 16, size=(M, size[c]))
+    scale = r.uniform(0.01, 2.0, g).astype(np.float32)
+    zero = r.integers(0, 16, g).astype(np.int32)
+    got = oracle.dequant_matmul_bf16(a, w, size, scale, zero, s_w)
+    xh = np.zeros((M, k_pad))
+    for c, (o, n_c) in enumerate(zip(off, size)):
+        xh[:, o:o + n_c] = _bf16_round(scale[c] * (a[:, o:o + n_c].astype(np.int32) - zero[c]).astype(np.float32))
+    want = (xh @ w.astype(np.float64).T) * s_w.astype(np.float64)
+    assert np.max(np.abs(got - want)) <= 1e-13 * np.abs(want).max()
+    # against the exact first method: every operand is off by at most 2^-9 of its magnitude
+    exact = oracle.dequant_matmul(a, w, size, scale.astype(np.float64), zero, s_w)
+    xe = np.zeros((M, k_pad))
+    for c, (o, n_c) in enumerate(zip(off, size)):
+        xe[:, o:o + n_c] = float(scale[c]) * (a[:, o:o + n_c].astype(np.float64) - zero[c])
+    bound = 2.0 ** -8 * (np.abs(xe) @ np.abs(w.astype(np.float64)).T) * s_w.astype(np.float64) + 1e-12
+    assert np.all(np.abs(got - exact) <= bound)
+    assert np.max(np.abs(got - exact)) > 0          # and the rounding is really there
