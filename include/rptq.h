@@ -183,6 +183,22 @@ int rptq_cluster_gemm(const rptq_layout_t* Lin, const void* a_codes, int M, cons
                       void* stream);
 
 /*
+ * Appendix, first computation method: de-quantise both operands, then one floating-point product,
+ *   X^ = s_c (X_q - z_c),  W^ = s_w[n] W_q,  y = X^ W^T  (+ bias[n]) (ReLU)
+ * as a bfloat16 tensor-core product with fp32 accumulation: X^ is formed in fp32 (one multiply of
+ * s_c with the exact integer difference) and rounded to bfloat16 in shared memory; the weight codes
+ * are exact in bfloat16 and s_w[n] multiplies the finished fp32 sum. One accumulator per output
+ * tile, no per-cluster accumulators: the workload for hardware or precisions where draining an
+ * accumulator per cluster costs more than the 16-bit product. Against the second method
+ * (rptq_cluster_gemm) the result differs by the bfloat16 rounding of X^ (2^-9 relative per operand).
+ * Arguments as for rptq_cluster_gemm (same packed activation codes and packed weights; wsum is not
+ * needed); y_dtype RPTQ_OUT_F32 or RPTQ_OUT_F16.
+ */
+int rptq_dequant_gemm(const rptq_layout_t* Lin, const void* a_codes, int M, const void* w_codes,
+                      const float* s_w, int64_t ld_w, const void* bias, int N, int act,
+                      void* y, int y_dtype, int64_t ldy, void* stream);
+
+/*
  * Appendix: "for one output channel, each weight cluster is quantised with its own asymmetric
  * parameters", W~_q,i = Q_k(W~_i, s^W_i, z^W_i), the paper's own weight scheme (it finds the codes
  * with GPTQ; here round-to-nearest). For output row r and input cluster c with n_c > 0, in fp32:

@@ -26,7 +26,7 @@ EXPORTS = (
     "rptq_weight_pack", "rptq_cluster_gemm", "rptq_cluster_gemm_debug_acc", "rptq_codes_unpack_host",
     "rptq_codes_pack_host", "rptq_weight_unpack_host", "rptq_get_device_status", "rptq_status_string",
     "rptq_format_version", "rptq_layout_padded_index", "rptq_weight_codes_bytes", "rptq_cluster_gemm_noalloc",
-    "rptq_ln_channel_minmax", "rptq_kmeans", "rptq_kmeans_workspace_bytes",
+    "rptq_dequant_gemm", "rptq_ln_channel_minmax", "rptq_kmeans", "rptq_kmeans_workspace_bytes",
     "rptq_probe_int8_peak", "rptq_weight_pack_clustered", "rptq_code_rowsums", "rptq_cluster_gemm_clustered",
 )
 
@@ -57,6 +57,7 @@ def _load(path: str = LIB_PATH) -> C.CDLL:
     lib.rptq_codes_pack_host.argtypes = [i32, i32, vp, i64, vp]
     lib.rptq_weight_unpack_host.argtypes = [i32, vp, i64, vp]
     lib.rptq_weight_codes_bytes.argtypes = [i32, i64]
+    lib.rptq_dequant_gemm.argtypes = [vp, vp, i32, vp, vp, i64, vp, i32, i32, vp, i32, i64, vp]
     lib.rptq_ln_channel_minmax.argtypes = [vp, i64, vp, vp, f32, i32, i32, vp, vp, vp]
     lib.rptq_kmeans_workspace_bytes.argtypes = [i32, i32]
     lib.rptq_kmeans.argtypes = [vp, i32, i32, i32, vp, i32, vp, vp, vp, vp, vp]
@@ -228,6 +229,16 @@ def cluster_gemm(layout_in: Layout, a_codes, M: int, w_codes, s_w, wsum, N: int,
                                   _dev_ptr(wsum), ld_w, _dev_ptr(bias), int(N), int(act),
                                   None if layout_out is None else layout_out.handle, _dev_ptr(y), int(y_dtype),
                                   int(ldy), _stream_ptr(stream)), "rptq_cluster_gemm")
+
+
+def dequant_gemm(layout_in: Layout, a_codes, M: int, w_codes, s_w, N: int, y, *, ld_w: Optional[int] = None, bias=None,
+                 act: int = ACT_NONE, y_dtype: int = OUT_F32, ldy: Optional[int] = None, stream=None) -> None:
+    """rptq_dequant_gemm on device tensors (the Appendix's first method as a bfloat16 product)."""
+    ld_w = int(s_w.shape[0]) if ld_w is None else int(ld_w)
+    ldy = int(y.stride(0)) if ldy is None else int(ldy)
+    _check(_lib.rptq_dequant_gemm(layout_in.handle, _dev_ptr(a_codes), int(M), _dev_ptr(w_codes), _dev_ptr(s_w), ld_w,
+                                  _dev_ptr(bias), int(N), int(act), _dev_ptr(y), int(y_dtype), int(ldy), _stream_ptr(stream)),
+           "rptq_dequant_gemm")
 
 
 def weight_pack_clustered(layout_in: Layout, W: np.ndarray, n_pad: Optional[int] = None):

@@ -107,6 +107,8 @@ struct Params {
     const int32_t* seg_cluster;
     const float* cl_n;
     const int32_t* xsum;
+    // first computation method (template mode MODE_DEQ): per unit of 32 positions {s_c, (float) z_c}
+    const float2* unit_sz;
     const float* bias;
     int act, y_dtype;
     void* y;
@@ -257,6 +259,26 @@ __device__ __forceinline__ void tc_mma_i8(uint32_t d_tmem, uint64_t a_desc, uint
             ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
     }
 }
+// bf16 x bf16 -> fp32, same operand layout and issue pattern as tc_mma_i8 (K = 16 elements = 32 bytes)
+template <int NCTA>
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    if constexpr (NCTA == 1) {
+        asm volatile(
+            "{\n\t.reg .pred p, q;\n\t"
+            "elect.sync _|q, 0xffffffff;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+    } else {
+        asm volatile(
+            "{\n\t.reg .pred p, q;\n\t"
+            "elect.sync _|q, 0xffffffff;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "@q tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+    }
+}
 __device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&v)[16])
 {
     asm volatile(
@@ -286,6 +308,49 @@ __host__ __device__ constexpr uint32_t instr_desc(int ncta)
     return (2u << 4) | (0u << 7) | (1u << 10) | ((uint32_t)(TILE_N >> 3) << 17) | ((uint32_t)((TILE_M * ncta) >> 4) << 24);
 }
 
+// kind::f16 with bfloat16 operands: D = fp32, A and B bfloat16, both K-major
+__host__ __device__ constexpr uint32_t instr_desc_bf16(int ncta)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(TILE_N >> 3) << 17) | ((uint32_t)((TILE_M * ncta) >> 4) << 24);
+}
+__device__ __forceinline__ float2 add2(float2 a, float2 b)
+{
+    float2 d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(reinterpret_cast<uint64_t&>(d))
+        : "l"(reinterpret_cast<uint64_t&>(a)), "l"(reinterpret_cast<uint64_t&>(b)));
+    return d;
+}
+__device__ __forceinline__ float2 mul2(float2 a, float2 b)
+{
+    float2 d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(reinterpret_cast<uint64_t&>(d))
+        : "l"(reinterpret_cast<uint64_t&>(a)), "l"(reinterpret_cast<uint64_t&>(b)));
+    return d;
+}
+// two fp32 values rounded to bfloat16 (nearest even): lo in bits 0-15, hi in bits 16-31
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
+{
+    uint32_t d;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+// Byte i of w as the float 2^23 + byte: the byte is dropped into the low mantissa bits of 0x4B000000.
+template <int I>
+__device__ __forceinline__ float byte_as_magic(uint32_t w)
+{
+    return __uint_as_float(__byte_perm(w, 0x4B000000u, 0x7650u | (uint32_t)I));
+}
+// Four 8-bit values of one word -> four bfloat16 (two words): v = (byte - c1) * s with c1 = 2^23 + z.
+// byte - c1 is exact, the product is rounded once to fp32 and once more to bfloat16.
+__device__ __forceinline__ void bytes_to_bf16(uint32_t w, float2 neg_c1, float2 s2, bool scale, uint32_t& out_lo, uint32_t& out_hi)
+{
+    float2 a = add2(make_float2(byte_as_magic<0>(w), byte_as_magic<1>(w)), neg_c1);
+    float2 b = add2(make_float2(byte_as_magic<2>(w), byte_as_magic<3>(w)), neg_c1);
+    if (scale) { a = mul2(a, s2); b = mul2(b, s2); }
+    out_lo = pack_bf16(a.x, a.y);
+    out_hi = pack_bf16(b.x, b.y);
+}
+
 // packed fp32 pairs: one instruction, two independent IEEE results
 __device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c)
 {
@@ -312,15 +377,23 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr)
 //   Y_q,c = acc'_c - (z^W_c[n] - 8) * sum_k X_q[m][k] - z^X_c * Wsum_c[n] + n_c z^X_c z^W_c[n] :
 // the first two are applied per element while a cluster's accumulator is drained, the last two are a
 // constant of the output column.
-template <int BITS, int NCTA, bool A8, bool ASYM>
+// MODE_DEQ: the first computation method of the Appendix (de-quantise, then one floating-point product):
+// the unpack warps write X^ = s_c (X_q - z_c) as bfloat16 and the weight codes as bfloat16 integers
+// (16 w, exact), the MMAs are kind::f16 into ONE fp32 accumulator per tile -- no per-cluster
+// accumulators, no drains at cluster boundaries -- and s_w[n] multiplies the finished sum. A bfloat16
+// operand row of 128 bytes holds 64 positions, so a K block of 128 positions is two operand stages.
+enum { MODE_INT = 0, MODE_ASYM = 1, MODE_DEQ = 2 };
+template <int BITS, int NCTA, bool A8, int MODE>
 __global__ void __launch_bounds__(THREADS, 1)
 cluster_gemm_kernel(const Params p)
 {
+    constexpr bool ASYM = MODE == MODE_ASYM, DEQ = MODE == MODE_DEQ;
+    static_assert(!(DEQ && A8), "the de-quantising variant unpacks every bit width");
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     constexpr SmemLayout SL = smem_layout(NCTA, BITS, A8);
     constexpr int W_ROWS = w_rows(NCTA);                 // weight rows this CTA stages and unpacks
     constexpr int N_P = n_p_stages(NCTA, BITS), N_U = n_u_stages(NCTA, A8);
-    constexpr uint32_t kInstrDesc = instr_desc(NCTA);
+    constexpr uint32_t kInstrDesc = DEQ ? instr_desc_bf16(NCTA) : instr_desc(NCTA);
     // dynamic shared memory is only guaranteed 16-byte alignment: round up to the swizzle span
     // (the offset is the same in both CTAs of a pair, as cta_group::2 descriptors require)
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -426,6 +499,34 @@ cluster_gemm_kernel(const Params p)
             uint32_t f4 = flags4[0];
             const uint32_t total_kb = (uint32_t)(((p.n_tiles - pair_id + n_pairs - 1) / n_pairs) * p.n_kb);
             int kb = 0;
+            if constexpr (DEQ) {
+                // One accumulator per tile, the two buffers alternate from tile to tile; every operand
+                // stage is half a K block (64 positions, four MMAs of K = 16).
+                const uint32_t steps_per_tile = 2u * (uint32_t)p.n_kb, total_steps = 2u * total_kb;
+                uint32_t in_tile = 0, b = 0;
+                for (uint32_t n = 0; n < total_steps; ++n) {
+                    const int st = n % N_U;
+                    if (in_tile == 0) {
+                        if (!mbar_wait_warp(bar(B_ACCEMPTY + b), ((par >> b) & 1u) ^ 1u, s_abort)) { ok = false; break; }
+                        tc_fence_after();
+                    }
+                    if (!mbar_wait_warp(bar(B_UFULL + st), (n / N_U) & 1, s_abort)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint64_t ad = a_desc0 + (uint64_t)(st * (SL.u_stage >> 4)), wd = ad + (uint64_t)(A8_BYTES >> 4);
+                    const uint32_t d_tmem = tmem_base + b * TILE_N;
+                    tc_mma_bf16<NCTA>(d_tmem, ad, wd, kInstrDesc, in_tile);
+                    tc_mma_bf16<NCTA>(d_tmem, ad + 2, wd + 2, kInstrDesc, 1u);
+                    tc_mma_bf16<NCTA>(d_tmem, ad + 4, wd + 4, kInstrDesc, 1u);
+                    tc_mma_bf16<NCTA>(d_tmem, ad + 6, wd + 6, kInstrDesc, 1u);
+                    tc_commit<NCTA>(bar(B_UEMPTY + st));
+                    if (++in_tile == steps_per_tile) {
+                        tc_commit<NCTA>(bar(B_ACCFULL + b));
+                        par ^= 1u << b;
+                        b ^= 1u;
+                        in_tile = 0;
+                    }
+                }
+            } else
             for (uint32_t n_kb_done = 0; n_kb_done < total_kb; ++n_kb_done) {
                     const int s = n_kb_done % N_U;
                     kb = kb + 1 == p.n_kb ? 0 : kb + 1;
@@ -620,6 +721,62 @@ cluster_gemm_kernel(const Params p)
                     for (int j = 0; j < BITS; ++j) pa_w[u][j] = raw[BITS * u + j];
             }
             if (!mbar_wait(bar(B_PFULL + sp), (n_done / N_P) & 1, s_abort)) break;
+            if constexpr (DEQ) {
+                // Two operand stages per K block, 64 positions each. My token row: units 2 h and 2 h + 1,
+                // de-quantised to bfloat16 with the unit's (s_c, z_c). Weights: for half h this thread
+                // converts unit 2 h + (ut & 1) of rows (ut >> 1) + 64 i.
+                const uint32_t pw = smem_base + SL.off_p + sp * SL.p_stage;
+                const int kb_now = it % p.n_kb;
+                bool ok = true;
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const uint32_t n_step = 2u * n_done + (uint32_t)h;
+                    const int st = n_step % N_U;
+                    if (!mbar_wait(bar(B_UEMPTY + st), ((n_step / N_U) & 1) ^ 1, s_abort)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_tile = smem_base + st * SL.u_stage, w_tile = a_tile + A8_BYTES;
+#pragma unroll
+                    for (int uu = 0; uu < 2; ++uu) {
+                        const int u = 2 * h + uu;
+                        const float2 sz = __ldg(p.unit_sz + 4 * kb_now + u);
+                        const float c1 = -(8388608.0f + sz.y);
+                        const float2 neg_c1 = make_float2(c1, c1), s2 = make_float2(sz.x, sz.x);
+                        uint32_t o[8];
+                        unpack_act32<BITS>(pa_w[u], o);
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            uint32_t b0, b1, b2, b3;
+                            bytes_to_bf16(o[2 * c], neg_c1, s2, true, b0, b1);
+                            bytes_to_bf16(o[2 * c + 1], neg_c1, s2, true, b2, b3);
+                            sts128(a_tile + a_off + (((4 * uu + c) ^ a_sw) << 4), b0, b1, b2, b3);
+                        }
+                    }
+                    const float cw = -(8388608.0f + 128.0f);
+                    const float2 neg_cw = make_float2(cw, cw);
+#pragma unroll
+                    for (int i = 0; i < W_ROWS / 64; ++i) {
+                        const int r = (ut >> 1) + 64 * i;
+                        const uint4 v = lds128(pw + r * 64 + (2 * h + (ut & 1)) * 16);
+                        const uint32_t pk[4] = {v.x, v.y, v.z, v.w};
+                        uint32_t o[8];
+                        unpack_w32_x16(pk, o);
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            uint32_t b0, b1, b2, b3;       // 16 w as bfloat16: the byte, sign bit flipped, minus 128
+                            bytes_to_bf16(o[2 * c] ^ 0x80808080u, neg_cw, neg_cw, false, b0, b1);
+                            bytes_to_bf16(o[2 * c + 1] ^ 0x80808080u, neg_cw, neg_cw, false, b2, b3);
+                            sts128(w_tile + r * 128 + (((4 * (ut & 1) + c) ^ (r & 7)) << 4), b0, b1, b2, b3);
+                        }
+                    }
+                    fence_proxy_async();
+                    __syncwarp();
+                    if (lane == 0) arrive_leader(bar(B_UFULL + st));
+                }
+                if (!ok) break;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(B_PEMPTY + sp));
+                continue;
+            }
             if (!mbar_wait(bar(B_UEMPTY + su), ((n_done / N_U) & 1) ^ 1, s_abort)) break;
             tc_fence_after();
             const uint32_t pw = smem_base + SL.off_p + sp * SL.p_stage;
@@ -676,6 +833,8 @@ cluster_gemm_kernel(const Params p)
                             corr = __fmaf_rn(s_cl_sz[c] * __ldg(p.sw_c + i), t, corr);
                         }
                         sw = 1.0f;
+                    } else if constexpr (DEQ) {
+                        sw = __ldg(p.s_w + n) * 0.0625f;             // the weight operands were 16 w; zero points are in X^
                     } else {
                         if (p.corr) corr = __ldg(p.corr + n);
                         else for (int c = 0; c < p.g; ++c) corr = __fmaf_rn(s_cl_sz[c], (float)__ldg(p.wsum + (int64_t)c * p.ld_w + n), corr);
@@ -689,8 +848,8 @@ cluster_gemm_kernel(const Params p)
             }
 #pragma unroll
             for (int i = 0; i < 64; ++i) R[i] = make_float2(0.f, 0.f);
-            for (int sgi = 0; sgi < p.n_seg; ++sgi) {
-                const uint32_t buf = s_seg_buf[sgi];
+            for (int sgi = 0; sgi < (DEQ ? 1 : p.n_seg); ++sgi) {
+                const uint32_t buf = DEQ ? (n_tile_done & 1u) : (uint32_t)s_seg_buf[sgi];
                 if (!mbar_wait(bar(B_ACCFULL + buf), (par >> buf) & 1u, s_abort)) { ok = false; break; }
                 par ^= 1u << buf;
                 tc_fence_after();
@@ -732,6 +891,9 @@ cluster_gemm_kernel(const Params p)
                                 r = __fmaf_rn(sx * sw4[e], t, r);
                             }
                         }
+                    } else if constexpr (DEQ) {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) R[c0 + i] = make_float2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));   // the fp32 sums themselves
                     } else {
 #pragma unroll
                         for (int i = 0; i < 8; ++i)
@@ -837,12 +999,12 @@ cluster_gemm_kernel(const Params p)
 }
 
 // ---------------------------------------------------------------- host side
-template <int BITS, int NCTA, bool A8, bool ASYM>
+template <int BITS, int NCTA, bool A8, int MODE>
 static int launch(const Params& p, int n_sm, cudaStream_t st)
 {
     constexpr SmemLayout SL = smem_layout(NCTA, BITS, A8);
     const int smem = SL.total + 1024;     // slack for the in-kernel 1024-byte alignment
-    const void* fn = reinterpret_cast<const void*>(cluster_gemm_kernel<BITS, NCTA, A8, ASYM>);
+    const void* fn = reinterpret_cast<const void*>(cluster_gemm_kernel<BITS, NCTA, A8, MODE>);
     cudaFuncAttributes attr;
     if (cudaFuncGetAttributes(&attr, fn) != cudaSuccess) return RPTQ_ERR_CUDA;
     // the register re-partition inside the kernel (setmaxnreg) assumes this pool; refuse to launch otherwise
@@ -860,7 +1022,7 @@ static int launch(const Params& p, int n_sm, cudaStream_t st)
     at[0].val.clusterDim.x = NCTA; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
     cfg.attrs = at;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, cluster_gemm_kernel<BITS, NCTA, A8, ASYM>, p) == cudaSuccess ? RPTQ_OK : RPTQ_ERR_CUDA;
+    return cudaLaunchKernelEx(&cfg, cluster_gemm_kernel<BITS, NCTA, A8, MODE>, p) == cudaSuccess ? RPTQ_OK : RPTQ_ERR_CUDA;
 }
 
 }  // namespace gemm
@@ -900,7 +1062,7 @@ static int launch_gemm(const rptq_layout_t* Lin, const void* a_codes, int M, con
                        const float* s_w, const int32_t* wsum, int64_t ld_w, const void* bias, int N,
                        int act, const rptq_layout_t* Lout, void* y, int y_dtype, int64_t ldy, void* stream,
                        int dev, int* status, const float* corr,
-                       const float* sw_c = nullptr, const int32_t* zw_c = nullptr, const int32_t* xsum = nullptr)
+                       const float* sw_c = nullptr, const int32_t* zw_c = nullptr, const int32_t* xsum = nullptr, bool deq = false)
 {
     gemm::Params p{};
     p.M = M; p.N = N; p.n_kb = Lin->K_pad / gemm::KBLK; p.n_seg = Lin->n_seg; p.g = Lin->g;
@@ -923,24 +1085,35 @@ static int launch_gemm(const rptq_layout_t* Lin, const void* a_codes, int M, con
     int n_sm = 0;
     if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return RPTQ_ERR_CUDA;
     auto st = static_cast<cudaStream_t>(stream);
+    if (deq) {
+        p.unit_sz = Lin->d_unit_sz;
+        if (ncta == 2) {
+            if (Lin->bits == 3) return gemm::launch<3, 2, false, gemm::MODE_DEQ>(p, n_sm, st);
+            if (Lin->bits == 4) return gemm::launch<4, 2, false, gemm::MODE_DEQ>(p, n_sm, st);
+            return gemm::launch<8, 2, false, gemm::MODE_DEQ>(p, n_sm, st);
+        }
+        if (Lin->bits == 3) return gemm::launch<3, 1, false, gemm::MODE_DEQ>(p, n_sm, st);
+        if (Lin->bits == 4) return gemm::launch<4, 1, false, gemm::MODE_DEQ>(p, n_sm, st);
+        return gemm::launch<8, 1, false, gemm::MODE_DEQ>(p, n_sm, st);
+    }
     if (sw_c) {
         if (ncta == 2) {
-            if (Lin->bits == 3) return gemm::launch<3, 2, false, true>(p, n_sm, st);
-            if (Lin->bits == 4) return gemm::launch<4, 2, false, true>(p, n_sm, st);
-            return gemm::launch<8, 2, true, true>(p, n_sm, st);
+            if (Lin->bits == 3) return gemm::launch<3, 2, false, gemm::MODE_ASYM>(p, n_sm, st);
+            if (Lin->bits == 4) return gemm::launch<4, 2, false, gemm::MODE_ASYM>(p, n_sm, st);
+            return gemm::launch<8, 2, true, gemm::MODE_ASYM>(p, n_sm, st);
         }
-        if (Lin->bits == 3) return gemm::launch<3, 1, false, true>(p, n_sm, st);
-        if (Lin->bits == 4) return gemm::launch<4, 1, false, true>(p, n_sm, st);
-        return gemm::launch<8, 1, false, true>(p, n_sm, st);
+        if (Lin->bits == 3) return gemm::launch<3, 1, false, gemm::MODE_ASYM>(p, n_sm, st);
+        if (Lin->bits == 4) return gemm::launch<4, 1, false, gemm::MODE_ASYM>(p, n_sm, st);
+        return gemm::launch<8, 1, false, gemm::MODE_ASYM>(p, n_sm, st);
     }
     if (ncta == 2) {
-        if (Lin->bits == 3) return gemm::launch<3, 2, false, false>(p, n_sm, st);
-        if (Lin->bits == 4) return gemm::launch<4, 2, false, false>(p, n_sm, st);
-        return gemm::launch<8, 2, true, false>(p, n_sm, st);      // 8-bit codes need no unpacking
+        if (Lin->bits == 3) return gemm::launch<3, 2, false, gemm::MODE_INT>(p, n_sm, st);
+        if (Lin->bits == 4) return gemm::launch<4, 2, false, gemm::MODE_INT>(p, n_sm, st);
+        return gemm::launch<8, 2, true, gemm::MODE_INT>(p, n_sm, st);      // 8-bit codes need no unpacking
     }
-    if (Lin->bits == 3) return gemm::launch<3, 1, false, false>(p, n_sm, st);
-    if (Lin->bits == 4) return gemm::launch<4, 1, false, false>(p, n_sm, st);
-    return gemm::launch<8, 1, false, false>(p, n_sm, st);
+    if (Lin->bits == 3) return gemm::launch<3, 1, false, gemm::MODE_INT>(p, n_sm, st);
+    if (Lin->bits == 4) return gemm::launch<4, 1, false, gemm::MODE_INT>(p, n_sm, st);
+    return gemm::launch<8, 1, false, gemm::MODE_INT>(p, n_sm, st);
 }
 
 extern "C" int rptq_cluster_gemm_clustered(const rptq_layout_t* Lin, const void* a_codes, int M, const int32_t* xsum,
@@ -971,6 +1144,23 @@ extern "C" int rptq_cluster_gemm(const rptq_layout_t* Lin, const void* a_codes, 
     int* status = device_status_word();
     if (!status) return RPTQ_ERR_ALLOC;
     return launch_gemm(Lin, a_codes, M, w_codes, s_w, wsum, ld_w, bias, N, act, Lout, y, y_dtype, ldy, stream, dev, status, nullptr);
+}
+
+extern "C" int rptq_dequant_gemm(const rptq_layout_t* Lin, const void* a_codes, int M, const void* w_codes,
+                                 const float* s_w, int64_t ld_w, const void* bias, int N, int act,
+                                 void* y, int y_dtype, int64_t ldy, void* stream)
+{
+    int dev = -1;
+    if (y_dtype != RPTQ_OUT_F32 && y_dtype != RPTQ_OUT_F16) return RPTQ_ERR_INVALID_ARG;
+    // (the integer tables of the second method are not needed: any aligned non-null pointer passes the shared checks)
+    const int rc = check_gemm_args(Lin, a_codes, M, w_codes, s_w, reinterpret_cast<const int32_t*>(s_w), ld_w, bias, N, act,
+                                   nullptr, y, y_dtype, ldy, &dev);
+    if (rc != RPTQ_OK) return rc;
+    if (M == 0) return RPTQ_OK;
+    int* status = device_status_word();
+    if (!status) return RPTQ_ERR_ALLOC;
+    return launch_gemm(Lin, a_codes, M, w_codes, s_w, nullptr, ld_w, bias, N, act, nullptr, y, y_dtype, ldy, stream, dev, status,
+                       nullptr, nullptr, nullptr, nullptr, true);
 }
 
 // ---------------------------------------------------------------- entry point that allocates nothing

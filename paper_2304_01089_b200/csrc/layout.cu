@@ -307,6 +307,10 @@ int rptq_layout_create(rptq_layout_t** out, int C, int g, int bits, const int32_
     if (rc == RPTQ_OK) rc = upload(&L->d_seg_buf, seg_buf.data(), seg_buf.size());
     if (rc == RPTQ_OK) rc = upload(&L->d_cl_n, cl_n.data(), cl_n.size());
     if (rc == RPTQ_OK) rc = upload(&L->d_seg_cluster, seg_cluster.data(), seg_cluster.size());
+    std::vector<float2> unit_sz((size_t)L->n_units, make_float2(1.0f, 0.0f));
+    for (int u = 0; u < L->n_units; ++u)
+        if (L->unit_cluster[u] >= 0) unit_sz[u] = make_float2(scale_host[L->unit_cluster[u]], (float)zero_host[L->unit_cluster[u]]);
+    if (rc == RPTQ_OK) rc = upload(&L->d_unit_sz, unit_sz.data(), unit_sz.size());
     if (rc == RPTQ_OK) rc = upload(&L->d_unit_cluster, L->unit_cluster.data(), L->unit_cluster.size());
     if (rc != RPTQ_OK) { rptq_layout_destroy(L); return rc; }
     *out = L;
@@ -342,6 +346,7 @@ int rptq_layout_destroy(rptq_layout_t* L)
     cudaFree(L->d_seg_buf);
     cudaFree(L->d_cl_n);
     cudaFree(L->d_seg_cluster);
+    cudaFree(L->d_unit_sz);
     cudaFree(L->d_unit_cluster);
     delete L;
     return RPTQ_OK;

@@ -50,6 +50,7 @@ struct rptq_layout {
     float* d_cl_sz = nullptr;           // [g]      s_c * z_c
     float* d_cl_n = nullptr;            // [g]      n_c
     int32_t* d_seg_cluster = nullptr;   // [n_seg]  the cluster of each entry of d_seg_scale
+    float2* d_unit_sz = nullptr;        // [n_units] {s_c, (float) z_c} of the unit's cluster ({1, 0} where there is none)
     int32_t* d_unit_cluster = nullptr;  // [n_units]
 };
 
