@@ -452,13 +452,15 @@ extern "C" int rptq_ln_reorder_quant(const rptq_layout_t* L, const void* x, int6
 
     // One gather thread per output unit where that fits beside four or five statistics warps in a
     // block of 512 threads (128 registers each), in up to four groups that take alternate rows when
-    // the layout is narrow; wider layouts get two statistics warps, and beyond 416
+    // the layout is narrow; wider layouts get two statistics warps (one beyond 416 units), and beyond 448
     // units each gather thread loops over several units and reloads its tables.
     const int want = (L->n_units + 31) / 32 * 32;
     int TG, S, groups = 1;
     if (want <= 320) { TG = want; S = 5; groups = 320 / TG; groups = groups > 4 ? 4 : groups; }
     else if (want <= 352) { TG = want; S = 4; }
-    else { TG = want <= 416 ? want : 416; S = 2; }
+    else if (want <= 416) { TG = want; S = 2; }
+    else if (want <= 448) { TG = want; S = 1; }        // one statistics warp keeps up with 14 gather warps on these long rows
+    else { TG = 416; S = 2; }
     if (groups > depth) groups = depth;
     const int T = 32 * (1 + S) + groups * TG;
 
