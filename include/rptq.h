@@ -329,6 +329,17 @@ int rptq_kmeans(const double* pts, int n, int dim, int g, const double* u, int i
  */
 int rptq_probe_int8_peak(int n_batches, int* failed_dev, double* ops_out, void* stream);
 
+/*
+ * Self-test of the give-up path of rptq_ln_reorder_quant (the paper has no counterpart): the same
+ * launch with every row's barrier told to expect 16 bytes more than its copy delivers and a wait
+ * budget of ten million cycles (~5 ms). The waits run out, RPTQ_ERR_DEVICE_TIMEOUT is recorded in the
+ * device's status word, the blocks drain and the kernel returns after some tens of milliseconds;
+ * `codes` (M rows of row_bytes bytes) receives undefined bytes. Nothing faults or spins without a
+ * limit; the context stays usable. Arguments as for rptq_ln_reorder_quant.
+ */
+int rptq_selftest_ln_timeout(const rptq_layout_t* L, const void* x, int64_t ldx, const void* gamma,
+                             const void* beta, float eps, int M, void* codes, void* stream);
+
 const char* rptq_status_string(int status);
 int rptq_format_version(void);
 

@@ -26,7 +26,7 @@ EXPORTS = (
     "rptq_weight_pack", "rptq_cluster_gemm", "rptq_cluster_gemm_debug_acc", "rptq_codes_unpack_host",
     "rptq_codes_pack_host", "rptq_weight_unpack_host", "rptq_get_device_status", "rptq_status_string",
     "rptq_format_version", "rptq_layout_padded_index", "rptq_weight_codes_bytes", "rptq_cluster_gemm_noalloc",
-    "rptq_dequant_gemm", "rptq_ln_channel_minmax", "rptq_kmeans", "rptq_kmeans_workspace_bytes",
+    "rptq_selftest_ln_timeout", "rptq_dequant_gemm", "rptq_ln_channel_minmax", "rptq_kmeans", "rptq_kmeans_workspace_bytes",
     "rptq_probe_int8_peak", "rptq_weight_pack_clustered", "rptq_code_rowsums", "rptq_cluster_gemm_clustered",
 )
 
@@ -57,6 +57,7 @@ def _load(path: str = LIB_PATH) -> C.CDLL:
     lib.rptq_codes_pack_host.argtypes = [i32, i32, vp, i64, vp]
     lib.rptq_weight_unpack_host.argtypes = [i32, vp, i64, vp]
     lib.rptq_weight_codes_bytes.argtypes = [i32, i64]
+    lib.rptq_selftest_ln_timeout.argtypes = [vp, vp, i64, vp, vp, f32, i32, vp, vp]
     lib.rptq_dequant_gemm.argtypes = [vp, vp, i32, vp, vp, i64, vp, i32, i32, vp, i32, i64, vp]
     lib.rptq_ln_channel_minmax.argtypes = [vp, i64, vp, vp, f32, i32, i32, vp, vp, vp]
     lib.rptq_kmeans_workspace_bytes.argtypes = [i32, i32]
@@ -195,6 +196,13 @@ def ln_reorder_quant(layout: Layout, x, gamma, beta, eps: float, codes, y_dbg=No
     _check(_lib.rptq_ln_reorder_quant(layout.handle, _dev_ptr(x), ldx, _dev_ptr(gamma), _dev_ptr(beta),
                                       C.c_float(eps), M, _dev_ptr(codes), _dev_ptr(y_dbg), _stream_ptr(stream)),
            "rptq_ln_reorder_quant")
+
+
+def selftest_ln_timeout(layout: Layout, x, gamma, beta, eps: float, codes, M: Optional[int] = None, stream=None) -> None:
+    """rptq_selftest_ln_timeout: the LayerNorm kernel with barriers that cannot complete and a ~5 ms wait budget."""
+    M = int(x.shape[0]) if M is None else int(M)
+    _check(_lib.rptq_selftest_ln_timeout(layout.handle, _dev_ptr(x), int(x.stride(0)), _dev_ptr(gamma), _dev_ptr(beta),
+                                         C.c_float(eps), M, _dev_ptr(codes), _stream_ptr(stream)), "rptq_selftest_ln_timeout")
 
 
 def weight_pack(layout_in: Layout, W: np.ndarray, out_perm=None, n_pad: Optional[int] = None):

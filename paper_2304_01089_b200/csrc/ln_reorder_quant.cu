@@ -89,7 +89,8 @@ constexpr long long kLnWaitBudgetCycles = 4000000000ll;   // about two seconds a
 // issue slots. When the budget runs out the status word is set, every later wait in the block
 // returns at once, and the caller carries on with whatever the slot holds: the loops have fixed
 // trip counts, so the kernel still ends.
-__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status)
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                          long long budget = kLnWaitBudgetCycles)
 {
     if (mbar_try_wait(bar, parity)) return;
     const long long t0 = clock64();
@@ -97,7 +98,7 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatil
     while (true) {
         if (mbar_try_wait_for(bar, parity, 4000u)) return;
         if (*abort_flag) return;
-        if (clock64() - t0 > kLnWaitBudgetCycles) {
+        if (clock64() - t0 > budget) {
             *abort_flag = 1;
             if (status) atomicExch(status, RPTQ_ERR_DEVICE_TIMEOUT);
             return;
@@ -112,6 +113,8 @@ struct LnParams {
     const int32_t* jidx_tab;     // [K_pad] reordered index of each padded position, -1 at pads (debug output)
     const UnitInfo* unit_tab;
     uint8_t* codes; int64_t row_bytes; float* y_dbg; int* status;
+    long long wait_budget;       // cycles a wait may take before the block gives up
+    uint32_t tx_extra;           // self-test only: bytes a row's barrier expects beyond what its copy delivers
 };
 
 // Warp roles:
@@ -189,10 +192,10 @@ ln_reorder_quant_kernel(const LnParams p)
             uint32_t par = 1;                // parity to wait for on free[d]: passes at once the first time round
             for (int k = 0; k < n_rows; ++k) {
                 // the gather threads have taken their gains and biases out of the last two slots
-                if (k == D - 2) mbar_wait(bar_s + 8 * (3 * D), 0u, s_abort, p.status);
-                mbar_wait(bar_s + 8 * (2 * D + d), par, s_abort, p.status);
+                if (k == D - 2) mbar_wait(bar_s + 8 * (3 * D), 0u, s_abort, p.status, p.wait_budget);
+                mbar_wait(bar_s + 8 * (2 * D + d), par, s_abort, p.status, p.wait_budget);
                 if (*s_abort) break;         // a wait ran out somewhere in the block: issue nothing more
-                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_s + 8 * d), "r"(row_bytes_in) : "memory");
+                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_s + 8 * d), "r"(row_bytes_in + p.tx_extra) : "memory");
                 asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                              ::"r"(ring_s + d * pitch), "l"(src), "r"(row_bytes_in), "r"(bar_s + 8 * d) : "memory");
                 src += row_step;
@@ -205,7 +208,8 @@ ln_reorder_quant_kernel(const LnParams p)
             if (*s_abort) {
                 for (int i = n_issued > D ? n_issued - D : 0; i < n_issued; ++i) {
                     const uint32_t b = bar_s + 8 * (i % D), ph = (uint32_t)(i / D) & 1u;
-                    for (int t = 0; t < (1 << 22) && !mbar_try_wait(b, ph); ++t) __nanosleep(64);
+                    const long long t0 = clock64();
+                    while (!mbar_try_wait_for(b, ph, 4000u) && clock64() - t0 <= p.wait_budget) {}
                 }
             }
         }
@@ -224,7 +228,7 @@ ln_reorder_quant_kernel(const LnParams p)
         const uint32_t zero_s = (uint32_t)__cvta_generic_to_shared(zero16);
         for (int k = warp - 1; k < n_rows; k += S) {
             const int d = k % D;
-            mbar_wait(bar_s + 8 * d, (uint32_t)(k / D) & 1u, s_abort, p.status);
+            mbar_wait(bar_s + 8 * d, (uint32_t)(k / D) & 1u, s_abort, p.status, p.wait_budget);
             const uint32_t row_s = ring_s + (uint32_t)d * pitch;
             float cs[4] = {0.f, 0.f, 0.f, 0.f}, qa[4] = {0.f, 0.f, 0.f, 0.f}, qb[4] = {0.f, 0.f, 0.f, 0.f};
             const uint32_t ones = 0x3C003C00u;       // two fp16 ones
@@ -335,7 +339,7 @@ ln_reorder_quant_kernel(const LnParams p)
         uint32_t par = 0;
         for (int k = 0; k < n_rows; ++k) {
             if (turn == grp) {
-                mbar_wait(bar_s + 8 * (D + d), par, s_abort, p.status);
+                mbar_wait(bar_s + 8 * (D + d), par, s_abort, p.status, p.wait_budget);
                 const float2 st = stats[d];
                 const float2 rs2 = make_float2(st.x, st.x), nm2 = make_float2(st.y, st.y);
                 const uint32_t slot = (uint32_t)d * pitch;
@@ -428,8 +432,8 @@ static int planned_blocks(const void* fn, int device, int T, size_t smem, int* b
 
 using namespace rptq;
 
-extern "C" int rptq_ln_reorder_quant(const rptq_layout_t* L, const void* x, int64_t ldx, const void* gamma,
-                                     const void* beta, float eps, int M, void* codes, float* y_dbg, void* stream)
+static int launch_ln(const rptq_layout_t* L, const void* x, int64_t ldx, const void* gamma, const void* beta, float eps,
+                     int M, void* codes, float* y_dbg, void* stream, long long wait_budget, uint32_t tx_extra)
 {
     if (!L || !x || !gamma || !beta || !codes) return RPTQ_ERR_INVALID_ARG;
     if (M < 0 || ldx < L->C || (ldx % 8) != 0 || !(eps >= 0.0f)) return RPTQ_ERR_INVALID_ARG;
@@ -473,6 +477,24 @@ extern "C" int rptq_ln_reorder_quant(const rptq_layout_t* L, const void* x, int6
     p.beta = static_cast<const __half*>(beta); p.eps = eps; p.M = M; p.C = C; p.n_units = L->n_units;
     p.n_stats_warps = S; p.depth = depth; p.n_groups = groups; p.ch_tab = L->d_src; p.jidx_tab = L->d_jidx; p.unit_tab = L->d_unit;
     p.codes = static_cast<uint8_t*>(codes); p.row_bytes = L->row_bytes; p.y_dbg = y_dbg; p.status = device_status_word();
+    p.wait_budget = wait_budget; p.tx_extra = tx_extra;
     fn<<<M < blocks ? M : blocks, T, smem, static_cast<cudaStream_t>(stream)>>>(p);
     return cudaGetLastError() == cudaSuccess ? RPTQ_OK : RPTQ_ERR_CUDA;
+}
+
+extern "C" int rptq_ln_reorder_quant(const rptq_layout_t* L, const void* x, int64_t ldx, const void* gamma,
+                                     const void* beta, float eps, int M, void* codes, float* y_dbg, void* stream)
+{
+    return launch_ln(L, x, ldx, gamma, beta, eps, M, codes, y_dbg, stream, kLnWaitBudgetCycles, 0u);
+}
+
+// Self-test of the give-up path: the same launch, but every row's barrier is told to expect 16 bytes
+// more than the row's copy delivers, so it never completes, and a wait may take 10 M cycles (~5 ms)
+// only. The statistics warps' waits run out, the block records RPTQ_ERR_DEVICE_TIMEOUT, every later
+// wait returns at once, the loops (fixed trip counts) run out and the kernel returns; nothing
+// faults and nothing spins without a limit. The codes it writes are undefined.
+extern "C" int rptq_selftest_ln_timeout(const rptq_layout_t* L, const void* x, int64_t ldx, const void* gamma,
+                                        const void* beta, float eps, int M, void* codes, void* stream)
+{
+    return launch_ln(L, x, ldx, gamma, beta, eps, M, codes, nullptr, stream, 10000000ll, 16u);
 }

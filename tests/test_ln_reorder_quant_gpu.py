@@ -227,3 +227,34 @@ def test_non_finite_inputs_still_give_in_range_codes():
     assert got.max() <= 15
     pads = L.padded_index() < 0
     assert not got[:, pads].any()
+
+
+def test_a_wait_that_runs_out_is_reported_and_the_next_launch_is_clean():
+    """The give-up path, made to happen without any fault: the library's self-test launch gives every
+    row's barrier an expectation that cannot be met and a ~5 ms budget. The kernel must come back, the
+    status word must read RPTQ_ERR_DEVICE_TIMEOUT exactly once, and an ordinary launch afterwards must
+    give the same bytes as one before."""
+    import time
+    import torch
+    from paper_2304_01089_b200 import binding
+    rng = np.random.default_rng(55)
+    C, M, bits = 1024, 600, 4
+    perm, size, scale, zero = random_layout_params(rng, C, 6, bits)
+    L = binding.Layout(perm, size, scale, zero, bits)
+    x = rng.normal(size=(M, C)).astype(np.float16)
+    gm = rng.lognormal(0, 0.3, C).astype(np.float16)
+    bt = rng.normal(size=C).astype(np.float16)
+    before, _ = _run(L, x, gm, bt, want_y=False)
+    xd, gd, bd = torch.from_numpy(x).cuda(), torch.from_numpy(gm).cuda(), torch.from_numpy(bt).cuda()
+    junk = torch.zeros((M + 1, L.row_bytes), dtype=torch.uint8, device="cuda")
+    junk[M] = CANARY
+    t0 = time.perf_counter()
+    binding.selftest_ln_timeout(L, xd, gd, bd, EPS, junk, M=M)
+    torch.cuda.synchronize()
+    assert time.perf_counter() - t0 < 5.0                       # it came back by itself
+    assert binding.get_device_status() == binding.ERR_DEVICE_TIMEOUT
+    assert binding.get_device_status() == 0                     # reading clears the word
+    assert bool((junk[M] == CANARY).all())                      # even the drained launch stays inside its rows
+    assert binding.status_string(binding.ERR_DEVICE_TIMEOUT) == "bounded wait inside a kernel ran out"
+    after, _ = _run(L, x, gm, bt, want_y=False)
+    assert np.array_equal(before, after)
