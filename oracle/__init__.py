@@ -315,6 +315,30 @@ def dequant_matmul_asym(a_codes, w_codes, size, scale, zero, s_w, z_w) -> np.nda
     return y
 
 
+# ---------------------------------------------------------------- attention sites (Sec. 4.2, 5.1)
+def attention(q_codes, k_codes, v_codes, H: int, gh: int, size_qk, sQ, zQ, sK, zK, size_v, sV, zV,
+              s_P: float, z_P: int, qk_scale: float, causal: bool, return_p: bool = False):
+    """Codes at padded positions: q [Tq][K_pad_qk], k [Tk][K_pad_qk], v [Tk][K_pad_v]; head h owns
+    clusters h*gh .. h*gh+gh-1 of both layouts. Returns O [Tq][K_pad_v] (and Pq [H][Tq][Tk])."""
+    q_codes, k_codes, v_codes = _arr(q_codes, np.uint8), _arr(k_codes, np.uint8), _arr(v_codes, np.uint8)
+    size_qk, size_v = _arr(size_qk, np.int32), _arr(size_v, np.int32)
+    sQ, sK, sV = _arr(sQ, np.float64), _arr(sK, np.float64), _arr(sV, np.float64)
+    zQ, zK, zV = _arr(zQ, np.int32), _arr(zK, np.int32), _arr(zV, np.int32)
+    Tq, kp = q_codes.shape
+    Tk, kpv = v_codes.shape
+    g = H * gh
+    assert k_codes.shape == (Tk, kp) and Tq <= Tk
+    for a in (size_qk, size_v, sQ, sK, sV, zQ, zK, zV):
+        assert a.shape == (g,)
+    out = np.empty((Tq, kpv))
+    pq = np.empty((H, Tq, Tk), np.uint8) if return_p else None
+    _lib.orc_attention(_p(q_codes), _p(k_codes), _p(v_codes), _i64(Tq), _i64(Tk), C.c_int(H), C.c_int(gh),
+                       _i32(kp), _p(size_qk), _p(sQ), _p(zQ), _p(sK), _p(zK),
+                       _i32(kpv), _p(size_v), _p(sV), _p(zV),
+                       _dbl(s_P), _i32(z_P), _dbl(qk_scale), C.c_int(1 if causal else 0), _p(out), _p(pq))
+    return (out, pq) if return_p else out
+
+
 # ---------------------------------------------------------------- calibration pipeline
 class Calibration(NamedTuple):
     perm: np.ndarray      # int32 [C]  reorder index S

@@ -743,3 +743,75 @@ void orc_dequant_matmul_bf16(const uint8_t* a_codes, int64_t M, const int8_t* w_
         }
     free(seg_off);
 }
+
+/* ------------------------------------------------------------------------------------------ */
+/* Attention sites (reorders R2 and R3)                                                        */
+/* ------------------------------------------------------------------------------------------ */
+
+/* Sec. 4.2: the query and the key of a head share one reorder index, so the products over the head's
+ * channels pair equal positions; Sec. 5.1: R2 and R3 are computed per head, every cluster has its own
+ * asymmetric parameters, and the softmax output is quantised at 8 bits. Self-attention of H heads on
+ * quantised Q, K and V, as its definition on the de-quantised operands (Eq. 1):
+ *   head h owns clusters h*gh .. h*gh + gh - 1 of both layouts (Q and K: size_qk; V: size_v);
+ *   Q^ = sQ_c (Qq - zQ_c), K^ = sK_c (Kq - zK_c), V^ = sV_c (Vq - zV_c) on the clusters' real positions;
+ *   A[i][j] = qk_scale * sum over the head's positions of Q^[i][p] K^[j][p];
+ *   key j is visible to query i when causal == 0 or j <= i + (Tk - Tq) (the queries are the last Tq
+ *   of the Tk tokens);
+ *   P[i][.] = softmax of A[i][.] over the visible keys, 0 at the hidden ones;
+ *   Pq = clamp(round_half_even(P / s_P) + z_P, 0, 255), P^ = s_P (Pq - z_P);
+ *   O[i][p] = sum_j P^[i][j] V^[j][p] for every real position p of the head in V's layout.
+ * Codes are given at padded positions (q, k: [T][K_pad_qk]; v: [Tk][K_pad_v]); out is [Tq][K_pad_v]
+ * with 0 at pad positions. p_codes, if not NULL, receives Pq as [H][Tq][Tk].
+ * The paper does not say where the 1/sqrt(d) of the scores is applied; it is a factor of the scores here. */
+void orc_attention(const uint8_t* q_codes, const uint8_t* k_codes, const uint8_t* v_codes,
+                   int64_t Tq, int64_t Tk, int H, int gh,
+                   int32_t K_pad_qk, const int32_t* size_qk, const double* sQ, const int32_t* zQ,
+                   const double* sK, const int32_t* zK,
+                   int32_t K_pad_v, const int32_t* size_v, const double* sV, const int32_t* zV,
+                   double s_P, int32_t z_P, double qk_scale, int causal, double* out, uint8_t* p_codes)
+{
+    const int g = H * gh;
+    int32_t* off_qk = (int32_t*)malloc(sizeof(int32_t) * (g + 1));
+    int32_t* off_v = (int32_t*)malloc(sizeof(int32_t) * (g + 1));
+    orc_segment_offsets(size_qk, g, off_qk);
+    orc_segment_offsets(size_v, g, off_v);
+    memset(out, 0, sizeof(double) * (size_t)Tq * (size_t)K_pad_v);
+#pragma omp parallel for schedule(dynamic, 4) collapse(2)
+    for (int h = 0; h < H; ++h)
+        for (int64_t i = 0; i < Tq; ++i) {
+            double* A = (double*)malloc(sizeof(double) * (size_t)Tk);
+            const int64_t last = causal ? i + (Tk - Tq) : Tk - 1;      /* last visible key */
+            double top = -INFINITY;
+            for (int64_t j = 0; j <= last; ++j) {
+                double a = 0.0;
+                for (int c = h * gh; c < (h + 1) * gh; ++c)
+                    for (int p = off_qk[c]; p < off_qk[c] + size_qk[c]; ++p) {
+                        const double qh = sQ[c] * ((double)q_codes[i * K_pad_qk + p] - (double)zQ[c]);
+                        const double kh = sK[c] * ((double)k_codes[j * K_pad_qk + p] - (double)zK[c]);
+                        a += qh * kh;
+                    }
+                A[j] = qk_scale * a;
+                if (A[j] > top) top = A[j];
+            }
+            double denom = 0.0;
+            for (int64_t j = 0; j <= last; ++j) denom += exp(A[j] - top);
+            for (int64_t j = 0; j < Tk; ++j) {
+                const double pr = j <= last ? exp(A[j] - top) / denom : 0.0;
+                double code = nearbyint(pr / s_P) + (double)z_P;       /* default rounding mode: half to even */
+                if (code < 0.0) code = 0.0;
+                if (code > 255.0) code = 255.0;
+                if (p_codes) p_codes[((int64_t)h * Tq + i) * Tk + j] = (uint8_t)code;
+                A[j] = s_P * (code - (double)z_P);                     /* P^ */
+            }
+            for (int c = h * gh; c < (h + 1) * gh; ++c)
+                for (int p = off_v[c]; p < off_v[c] + size_v[c]; ++p) {
+                    double o = 0.0;
+                    for (int64_t j = 0; j < Tk; ++j)
+                        o += A[j] * (sV[c] * ((double)v_codes[j * K_pad_v + p] - (double)zV[c]));
+                    out[i * K_pad_v + p] = o;
+                }
+            free(A);
+        }
+    free(off_qk);
+    free(off_v);
+}

@@ -821,6 +821,9 @@ cluster_gemm_kernel(const Params p)
         for (int t = pair_id; t < p.n_tiles && ok; t += n_pairs, ++n_tile_done) {
             const int m0 = (t % p.tiles_m) * (TILE_M * NCTA) + (int)cta_rank * TILE_M, n0 = (t / p.tiles_m) * TILE_N;
             float* tab = s_tab + (n_tile_done & 1) * 3 * TILE_N;
+            // a warp whose 32 accumulator lanes all lie beyond the last token row keeps the barriers'
+            // protocol but reads and accumulates nothing (few-token calls: most of the tile is empty)
+            const bool live = m0 + 32 * q < p.M;
             {   // per-tile column constants: zero-point correction sum_c s_c z_c Wsum_c[n], s_w[n], bias[n]
                 const int n = n0 + et;
                 float corr = 0.f, sw = 0.f, bs = 0.f;
@@ -856,6 +859,7 @@ cluster_gemm_kernel(const Params p)
                 const float sc = s_seg_scale[sgi];
                 const float2 sc2 = make_float2(sc, sc);
                 const uint32_t taddr = tmem_base + ((uint32_t)(32 * q) << 16) + buf * TILE_N + h * 128;
+                if (live) {
                 uint32_t va[16], vb[16];
                 tc_ld16(taddr, va);
                 // ASYM: this cluster's row of the weight tables and my token's code sum
@@ -909,6 +913,7 @@ cluster_gemm_kernel(const Params p)
                     if (ch + 2 < 8) tc_ld16(taddr + (ch + 2) * 16, va);
                     accumulate(vb, (ch + 1) * 8);
                 }
+                }
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) arrive_leader(bar(B_ACCEMPTY + buf));
@@ -922,11 +927,13 @@ cluster_gemm_kernel(const Params p)
             const float* t_sw = tab + TILE_N + h * 128;
             const float* t_bs = tab + 2 * TILE_N + h * 128;
             auto Rf = [&](int i) -> float& { return (i & 1) ? R[i >> 1].y : R[i >> 1].x; };
+            if (live) {
 #pragma unroll
-            for (int i = 0; i < 128; ++i) {
-                float v = __fmaf_rn(t_sw[i], Rf(i) - t_corr[i], t_bs[i]);
-                if (p.act == RPTQ_ACT_RELU) v = fmaxf(v, 0.f);
-                Rf(i) = v;
+                for (int i = 0; i < 128; ++i) {
+                    float v = __fmaf_rn(t_sw[i], Rf(i) - t_corr[i], t_bs[i]);
+                    if (p.act == RPTQ_ACT_RELU) v = fmaxf(v, 0.f);
+                    Rf(i) = v;
+                }
             }
             if (m < p.M) {
                 if (p.y_dtype == RPTQ_OUT_F32) {

@@ -590,3 +590,117 @@ def test_bf16_first_method_against_numpy_and_within_its_rounding_bound():
     bound = 2.0 ** -8 * (np.abs(xe) @ np.abs(w.astype(np.float64)).T) * s_w.astype(np.float64) + 1e-12
     assert np.all(np.abs(got - exact) <= bound)
     assert np.max(np.abs(got - exact)) > 0          # and the rounding is really there
+
+
+# ------------------------------------------------------------------ attention sites (Sec. 4.2, 5.1)
+def _toy_attention(causal):
+    q = np.zeros((2, 128), np.uint8); k = np.zeros((2, 128), np.uint8); v = np.zeros((2, 128), np.uint8)
+    q[0, 0:2] = (4, 2); q[0, 32] = 1; q[1, 0:2] = (6, 0); q[1, 32] = 1
+    k[0, 0:2] = (2, 3); k[0, 32] = 5; k[1, 0:2] = (3, 1); k[1, 32] = 3
+    v[0, 0] = 8; v[0, 32:34] = (3, 0); v[1, 0] = 0; v[1, 32:34] = (1, 2)
+    return oracle.attention(q, k, v, 1, 2, [2, 1], [0.5, 2.0], [2, 0], [1.0, 0.5], [1, 3], [1, 2], [0.25, 2.0], [4, 1],
+                            1.0 / 256, 0, np.log(3.0) / 2, causal, return_p=True)
+
+
+def test_attention_hand_worked_example():
+    n = 0
+    for line in _golden_rows("attention_toy.txt"):
+        kind, pq_want, o_want = [p.strip() for p in line.split("|")]
+        o, pq = _toy_attention(kind == "causal")
+        assert pq.reshape(-1).tolist() == [int(t) for t in pq_want.split()]
+        got = np.concatenate([o[:, 0:1], o[:, 32:34]], axis=1).reshape(-1)
+        assert np.allclose(got, [float(t) for t in o_want.split()], rtol=0, atol=1e-15)
+        assert not o[:, 1:32].any() and not o[:, 34:].any()         # pad positions stay 0
+        n += 1
+    assert n == 2
+
+
+def _attention_case(seed, Tq=5, Tk=9, H=2, gh=3, hd=24, bits=4):
+    r = _rng(seed)
+    def sizes():
+        out = []
+        for _ in range(H):
+            cuts = np.sort(r.integers(0, hd + 1, size=gh - 1))
+            out.append(np.diff(np.concatenate([[0], cuts, [hd]])))
+        return np.concatenate(out).astype(np.int32)
+    size_qk, size_v = sizes(), sizes()
+    g = H * gh
+    par = lambda: (r.uniform(0.05, 0.3, size=g), r.integers(0, 1 << bits, size=g).astype(np.int32))
+    (sQ, zQ), (sK, zK), (sV, zV) = par(), par(), par()
+    def codes(T, size):
+        off, k_pad = oracle.segment_offsets(size)
+        a = np.zeros((T, k_pad), np.uint8)
+        for c in range(g):
+            a[:, off[c]:off[c] + size[c]] = r.integers(0, 1 << bits, size=(T, size[c]))
+        return a, off
+    (q, off_qk), (k, _), (v, off_v) = codes(Tq, size_qk), codes(Tk, size_qk), codes(Tk, size_v)
+    return dict(q=q, k=k, v=v, H=H, gh=gh, size_qk=size_qk, sQ=sQ, zQ=zQ, sK=sK, zK=zK, size_v=size_v, sV=sV, zV=zV,
+                off_qk=off_qk, off_v=off_v, hd=hd)
+
+
+def _dequant_by_hand(codes, off, size, s, z):
+    """Eq. 1 on the real positions of every cluster; other positions 0."""
+    out = np.zeros(codes.shape)
+    for c in range(len(size)):
+        sl = slice(off[c], off[c] + size[c])
+        out[:, sl] = s[c] * (codes[:, sl].astype(np.float64) - z[c])
+    return out
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_attention_is_within_the_softmax_quantisers_bound_of_plain_attention(causal):
+    """With the 8-bit softmax output replaced by the exact probabilities the computation is ordinary
+    attention on the de-quantised tensors (scipy's softmax); the quantiser moves a probability by at most
+    s_P / 2 (plus the clamp of 256 to 255), so |O - O_exact| <= (s_P / 2 + s_P [P = 1]) sum_j |V^|."""
+    from scipy.special import softmax
+    for seed in (1, 2, 3):
+        c = _attention_case(seed)
+        Tq, Tk, H, gh = c["q"].shape[0], c["k"].shape[0], c["H"], c["gh"]
+        scale = 1.0 / np.sqrt(c["hd"])
+        o, pq = oracle.attention(c["q"], c["k"], c["v"], H, gh, c["size_qk"], c["sQ"], c["zQ"], c["sK"], c["zK"],
+                                 c["size_v"], c["sV"], c["zV"], 1.0 / 256, 0, scale, causal, return_p=True)
+        Qh = _dequant_by_hand(c["q"], c["off_qk"], c["size_qk"], c["sQ"], c["zQ"])
+        Kh = _dequant_by_hand(c["k"], c["off_qk"], c["size_qk"], c["sK"], c["zK"])
+        Vh = _dequant_by_hand(c["v"], c["off_v"], c["size_v"], c["sV"], c["zV"])
+        for h in range(H):
+            lo, hi = c["off_qk"][h * gh], c["off_qk"][(h + 1) * gh]
+            A = scale * Qh[:, lo:hi] @ Kh[:, lo:hi].T
+            if causal:
+                A = np.where(np.arange(Tk)[None, :] <= np.arange(Tq)[:, None] + (Tk - Tq), A, -np.inf)
+            P = softmax(A, axis=1)
+            vlo, vhi = c["off_v"][h * gh], c["off_v"][(h + 1) * gh]
+            exact = P @ Vh[:, vlo:vhi]
+            bound = (1.5 / 256) * np.abs(Vh[:, vlo:vhi]).sum(axis=0)[None, :] + 1e-12
+            assert np.all(np.abs(o[:, vlo:vhi] - exact) <= bound)
+            assert np.abs(o[:, vlo:vhi] - exact).max() > 0                      # and the quantiser is really there
+            assert np.all(np.abs(pq[h].astype(np.float64) - np.minimum(np.rint(P * 256), 255)) <= 1)
+            if causal:
+                assert not pq[h][np.arange(Tk)[None, :] > np.arange(Tq)[:, None] + (Tk - Tq)].any()
+
+
+def test_attention_closed_forms():
+    c = _attention_case(7, Tq=4, Tk=6)
+    H, gh = c["H"], c["gh"]
+    Vh = _dequant_by_hand(c["v"], c["off_v"], c["size_v"], c["sV"], c["zV"])
+    args = lambda k, s: (c["q"], k, c["v"], H, gh, c["size_qk"], c["sQ"], c["zQ"], c["sK"], c["zK"], c["size_v"], c["sV"], c["zV"],
+                         1.0 / 256, 0, s, False)
+    # equal keys: every probability is 1/6 -> code round(256 / 6) = 43, O = 43/256 sum_j V^
+    k_same = np.repeat(c["k"][:1], 6, axis=0)
+    o, pq = oracle.attention(*args(k_same, 0.3), return_p=True)
+    assert np.all(pq == 43)
+    assert np.allclose(o, np.broadcast_to((43.0 / 256) * Vh.sum(axis=0), o.shape), rtol=0, atol=1e-12)
+    # a score scale of 0 does the same whatever the keys are
+    assert np.array_equal(oracle.attention(*args(c["k"], 0.0)), o)
+    # a zero point of the softmax codes cancels in s_P (Pq - z_P) as long as nothing clamps
+    a = list(args(k_same, 0.3)); a[14] = 100
+    assert np.allclose(oracle.attention(*a), o, rtol=0, atol=1e-12)
+    # a huge score scale picks, per query and head, the key with the largest product: P = 1 -> 255/256 V^[j*]
+    o, pq = oracle.attention(*args(c["k"], 1e4), return_p=True)
+    Qh = _dequant_by_hand(c["q"], c["off_qk"], c["size_qk"], c["sQ"], c["zQ"])
+    Kh = _dequant_by_hand(c["k"], c["off_qk"], c["size_qk"], c["sK"], c["zK"])
+    for h in range(H):
+        lo, hi = c["off_qk"][h * gh], c["off_qk"][(h + 1) * gh]
+        best = np.argmax(Qh[:, lo:hi] @ Kh[:, lo:hi].T, axis=1)
+        vlo, vhi = c["off_v"][h * gh], c["off_v"][(h + 1) * gh]
+        assert np.allclose(o[:, vlo:vhi], (255.0 / 256) * Vh[best, vlo:vhi], rtol=0, atol=1e-12)
+        assert np.all(pq[h][np.arange(4), best] == 255) and pq[h].sum() == 4 * 255
