@@ -340,6 +340,35 @@ int rptq_probe_int8_peak(int n_batches, int* failed_dev, double* ops_out, void* 
 int rptq_selftest_ln_timeout(const rptq_layout_t* L, const void* x, int64_t ldx, const void* gamma,
                              const void* beta, float eps, int M, void* codes, void* stream);
 
+/*
+ * Sec. 4.2 and 5.1: self-attention on quantised Q, K and V. The query and the key of a head are
+ * multiplied position by position, so they share one reorder index (their channels are clustered
+ * together, on the points (Q max, Q min, K max, K min)); the attention sites are reordered per
+ * head; the softmax output is quantised at 8 bits. For head h, query i, key j:
+ *   A[i][j]  = qk_scale * sum_c s^Q_c s^K_c sum_{p in c} (Q_q[i][p] - z^Q_c)(K_q[j][p] - z^K_c)
+ *              (integer products per cluster segment of the head on the tensor cores, fp32 scaling)
+ *   key j is visible to query i when causal == 0 or j <= i + (Tk - Tq)
+ *   P        = softmax of A over the visible keys (fp32),  P_q = min(rne(P / s_P), 255)
+ *   O[i][ch] = s_P s^V_c (sum_j P_q[i][j] V_q[j][p] - z^V_c sum_j P_q[i][j])   for V's position p of channel ch
+ *              (integer sums, exact), written as fp16.
+ * Layouts: LQ, LK, LV have n_heads * (clusters per head) clusters in RPTQ_ORDER_CONTIGUOUS order, head h
+ * owning clusters h * g / n_heads .. (h + 1) * g / n_heads - 1 and the channels h * d .. (h + 1) * d - 1;
+ * LQ and LK must have the same reorder index and cluster sizes (their scales and zero points differ).
+ * A head may take at most 8 units of 32 positions in LQ / LK.
+ *   q_codes  dev, Tq rows of LQ.row_bytes bytes (as an RPTQ_OUT_CODES GEMM writes them)
+ *   k_codes, v_codes  dev, Tk rows of LK.row_bytes / LV.row_bytes bytes: the quantised key / value cache
+ *   s_P, z_P Eq. 1 parameters of the softmax output for codes in [0, 255]; z_P must be 0 (Eq. 2 on a
+ *            range that starts at 0 gives exactly that), otherwise RPTQ_ERR_UNSUPPORTED
+ *   out_f16  dev fp16 [Tq][ldo], ldo >= LV.C: channel ch of token i at out[i * ldo + ch]
+ *   p_codes_out  NULL, or dev uint8 [n_heads][Tq][Tk]: receives P_q at the visible keys of key tiles
+ *            that hold a visible key (a test aid; clear it before the call)
+ * Tk >= Tq; Tk * 255 * 255 < 2^31. Row-constant terms of A cancel in the softmax and are not formed.
+ */
+int rptq_attention(const rptq_layout_t* LQ, const rptq_layout_t* LK, const rptq_layout_t* LV, int n_heads,
+                   const void* q_codes, int Tq, const void* k_codes, const void* v_codes, int Tk,
+                   float s_P, int z_P, float qk_scale, int causal,
+                   void* out_f16, int64_t ldo, uint8_t* p_codes_out, void* stream);
+
 const char* rptq_status_string(int status);
 int rptq_format_version(void);
 

@@ -339,6 +339,18 @@ def attention(q_codes, k_codes, v_codes, H: int, gh: int, size_qk, sQ, zQ, sK, z
     return (out, pq) if return_p else out
 
 
+def attention_output(p_codes, v_codes, H: int, gh: int, size_v, sV, zV, s_P: float, z_P: int) -> np.ndarray:
+    """O from given softmax codes p_codes [H][Tq][Tk] and V codes [Tk][K_pad_v]."""
+    p_codes, v_codes = _arr(p_codes, np.uint8), _arr(v_codes, np.uint8)
+    size_v, sV, zV = _arr(size_v, np.int32), _arr(sV, np.float64), _arr(zV, np.int32)
+    Hn, Tq, Tk = p_codes.shape
+    assert Hn == H and v_codes.shape[0] == Tk and size_v.shape == (H * gh,)
+    out = np.empty((Tq, v_codes.shape[1]))
+    _lib.orc_attention_output(_p(p_codes), _p(v_codes), _i64(Tq), _i64(Tk), C.c_int(H), C.c_int(gh), _i32(v_codes.shape[1]),
+                              _p(size_v), _p(sV), _p(zV), _dbl(s_P), _i32(z_P), _p(out))
+    return out
+
+
 # ---------------------------------------------------------------- calibration pipeline
 class Calibration(NamedTuple):
     perm: np.ndarray      # int32 [C]  reorder index S

@@ -815,3 +815,28 @@ void orc_attention(const uint8_t* q_codes, const uint8_t* k_codes, const uint8_t
     free(off_qk);
     free(off_v);
 }
+
+/* The last step of orc_attention alone, on given softmax codes (p_codes [H][Tq][Tk]):
+ *   O[i][p] = sum_j s_P (Pq[i][j] - z_P) sV_c (Vq[j][p] - zV_c)
+ * for comparing an implementation whose softmax codes differ from orc_attention's by a rounding. */
+void orc_attention_output(const uint8_t* p_codes, const uint8_t* v_codes, int64_t Tq, int64_t Tk, int H, int gh,
+                          int32_t K_pad_v, const int32_t* size_v, const double* sV, const int32_t* zV,
+                          double s_P, int32_t z_P, double* out)
+{
+    const int g = H * gh;
+    int32_t* off_v = (int32_t*)malloc(sizeof(int32_t) * (g + 1));
+    orc_segment_offsets(size_v, g, off_v);
+    memset(out, 0, sizeof(double) * (size_t)Tq * (size_t)K_pad_v);
+#pragma omp parallel for schedule(dynamic, 4) collapse(2)
+    for (int h = 0; h < H; ++h)
+        for (int64_t i = 0; i < Tq; ++i)
+            for (int c = h * gh; c < (h + 1) * gh; ++c)
+                for (int p = off_v[c]; p < off_v[c] + size_v[c]; ++p) {
+                    double o = 0.0;
+                    for (int64_t j = 0; j < Tk; ++j)
+                        o += s_P * ((double)p_codes[((int64_t)h * Tq + i) * Tk + j] - (double)z_P) *
+                             (sV[c] * ((double)v_codes[j * K_pad_v + p] - (double)zV[c]));
+                    out[i * K_pad_v + p] = o;
+                }
+    free(off_v);
+}

@@ -611,6 +611,11 @@ def test_attention_hand_worked_example():
         got = np.concatenate([o[:, 0:1], o[:, 32:34]], axis=1).reshape(-1)
         assert np.allclose(got, [float(t) for t in o_want.split()], rtol=0, atol=1e-15)
         assert not o[:, 1:32].any() and not o[:, 34:].any()         # pad positions stay 0
+        # the last step alone, from the fixture's codes
+        v = np.zeros((2, 128), np.uint8); v[0, 0] = 8; v[0, 32:34] = (3, 0); v[1, 32:34] = (1, 2)
+        o2 = oracle.attention_output(np.array([int(t) for t in pq_want.split()], np.uint8).reshape(1, 2, 2), v, 1, 2,
+                                     [1, 2], [0.25, 2.0], [4, 1], 1.0 / 256, 0)
+        assert np.allclose(np.concatenate([o2[:, 0:1], o2[:, 32:34]], axis=1).reshape(-1), [float(t) for t in o_want.split()], rtol=0, atol=1e-15)
         n += 1
     assert n == 2
 
