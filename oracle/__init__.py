@@ -387,3 +387,35 @@ def calibrate(x_cal16, gamma16, beta16, g: int, k: int, u, eps: float = 1e-5, it
     y = layernorm(x_cal16, gamma16, beta16, eps)
     x_min, x_max = channel_minmax(y)
     return calibrate_from_minmax(x_min, x_max, g, k, u, iters)
+
+
+def calibrate_heads(ranges, n_heads: int, g_head: int, bits, u, iters: int = 20):
+    """Sec. 4.2 / 5.1: per-head reorder of an attention site. `ranges`: [(min, max)] per tensor that shares
+    the index -- for Q and K the head's channels are clustered on the 4-D points (Q max, Q min, K max,
+    K min). Composition of orc_kmeans, orc_reorder_index (on the union of the ranges) and
+    orc_minmax_params per tensor and cluster. Returns (perm, size, [scale per tensor], [zero per tensor])."""
+    ranges = [(_arr(lo, np.float64), _arr(hi, np.float64)) for lo, hi in ranges]
+    Cn = ranges[0][0].shape[0]
+    d = Cn // n_heads
+    lo_all = np.min([r[0] for r in ranges], axis=0)
+    hi_all = np.max([r[1] for r in ranges], axis=0)
+    perm, size = [], []
+    scale = [[] for _ in ranges]
+    zero = [[] for _ in ranges]
+    for h in range(n_heads):
+        sl = slice(h * d, (h + 1) * d)
+        pts = np.stack([a[sl] for r in ranges for a in (r[1], r[0])], axis=1)
+        labels, _, _ = kmeans(pts, g_head, np.asarray(u)[h], iters)
+        p_h, size_h, _ = reorder_index(labels, lo_all[sl], hi_all[sl], g_head)
+        perm.append(h * d + p_h)
+        size.append(size_h)
+        pos = 0
+        for c in range(g_head):
+            n = int(size_h[c])
+            seg = h * d + p_h[pos:pos + n]
+            for t, (lo, hi) in enumerate(ranges):
+                s, z = minmax_params(lo[seg].min(), hi[seg].max(), bits[t]) if n else (1.0, 1 << (bits[t] - 1))
+                scale[t].append(s); zero[t].append(z)
+            pos += n
+    return (np.concatenate(perm).astype(np.int32), np.concatenate(size).astype(np.int32),
+            [np.array(x, np.float64) for x in scale], [np.array(x, np.int32) for x in zero])

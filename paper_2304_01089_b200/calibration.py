@@ -173,6 +173,65 @@ def calibrate_on_device(x_cal, gamma, beta, g: int, k: int, draws, eps: float = 
     return calibrate_from_minmax(x_min.cpu().numpy(), x_max.cpu().numpy(), g, k, draws, iters, labels=labels.cpu().numpy())
 
 
+class HeadCalibration(NamedTuple):
+    """Per-head reorder of an attention site: head h owns channels h*d .. (h+1)*d - 1 and clusters
+    h*g_head .. (h+1)*g_head - 1. One (scale, zero) pair per tensor that shares the index."""
+    perm: np.ndarray      # int32 [H*d]
+    size: np.ndarray      # int32 [H*g_head]
+    scale: tuple          # of fp32 [H*g_head]
+    zero: tuple           # of int32 [H*g_head]
+
+
+def _kmeans_host_or_device(points: np.ndarray, g: int, draws, iters: int, device):
+    if device is None:
+        return kmeans(points, g, draws, iters)[0]
+    import torch
+    from . import binding
+    n, dim = points.shape
+    pts = torch.from_numpy(np.ascontiguousarray(points, dtype=np.float64)).to(device)
+    u = torch.from_numpy(np.ascontiguousarray(draws, dtype=np.float64)).to(device)
+    labels = torch.empty(n, dtype=torch.int32, device=device)
+    centres = torch.empty((g, dim), dtype=torch.float64, device=device)
+    work = torch.empty(binding.kmeans_workspace_bytes(n, g), dtype=torch.uint8, device=device)
+    binding.kmeans(pts, g, u, iters, labels, centres, None, work)
+    return labels.cpu().numpy()
+
+
+def calibrate_heads(ranges, n_heads: int, g_head: int, bits, draws, iters: int = 20, device=None) -> HeadCalibration:
+    """Sec. 4.2 / 5.1: the reorder of an attention site, computed per head. `ranges` is a list of
+    (x_min, x_max) pairs, one per tensor that must share the index: [(Q), (K)] for R2 -- the head's
+    channels are clustered on the points (Q max, Q min, K max, K min) -- and [(V)] for R3. Every tensor
+    gets its own Min-Max parameters per cluster (Eq. 2) with its own bit width bits[t]. draws: [H][g_head]
+    uniform numbers for the K-Means seeding. device: a torch device to run the K-Means there (rptq_kmeans).
+    The clusters of a head are ordered by the union of the tensors' ranges."""
+    ranges = [(np.asarray(lo, np.float64), np.asarray(hi, np.float64)) for lo, hi in ranges]
+    Cn = ranges[0][0].shape[0]
+    d = Cn // n_heads
+    assert d * n_heads == Cn and len(bits) == len(ranges)
+    lo_all = np.min([r[0] for r in ranges], axis=0)
+    hi_all = np.max([r[1] for r in ranges], axis=0)
+    perm, size = [], []
+    scale = [[] for _ in ranges]
+    zero = [[] for _ in ranges]
+    for h in range(n_heads):
+        sl = slice(h * d, (h + 1) * d)
+        pts = np.stack([a[sl] for r in ranges for a in (r[1], r[0])], axis=1)      # (max, min) per tensor
+        labels = _kmeans_host_or_device(pts, g_head, np.asarray(draws)[h], iters, device)
+        p_h, size_h, _ = reorder_index(np.asarray(labels), lo_all[sl], hi_all[sl], g_head)
+        perm.append(h * d + p_h)
+        size.append(size_h)
+        pos = 0
+        for c in range(g_head):
+            n = int(size_h[c])
+            seg = h * d + p_h[pos:pos + n]
+            for t, (lo, hi) in enumerate(ranges):
+                s, z = minmax_params(lo[seg].min(), hi[seg].max(), bits[t]) if n else (1.0, 1 << (bits[t] - 1))
+                scale[t].append(np.float32(s)); zero[t].append(z)
+            pos += n
+    return HeadCalibration(np.concatenate(perm).astype(np.int32), np.concatenate(size).astype(np.int32),
+                           tuple(np.array(s, np.float32) for s in scale), tuple(np.array(z, np.int32) for z in zero))
+
+
 def segment_offsets(size: np.ndarray):
     """Padded segment layout of the library: segments start at multiples of 32, rows are a
     multiple of 128 long. Returns (seg_off int32 [g+1], K_pad)."""

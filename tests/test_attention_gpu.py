@@ -189,3 +189,58 @@ def test_opt66b_heads_sampled_rows():
         vmax = float(c.sV[cl].max()) * 15
         assert np.all(np.abs(got - w) <= 8 * c.s_P * vmax + 1.01 * FP16 * np.abs(w) + 1e-7)
         assert np.abs(got - w).max() <= 0.05 * np.abs(w).max() + 8 * c.s_P * vmax
+
+
+def test_projections_write_the_cache_and_attention_reads_it():
+    """Sec. 4.2: the Q, K and V projections' rows follow the attention sites' reorder indices, so their
+    epilogues write the quantised query and the quantised key / value cache directly (RPTQ_OUT_CODES); the
+    indices come from the per-head calibration with the K-Means on the device (Q and K clustered together
+    on 4-D points). rptq_attention on those buffers against the oracle on the same codes."""
+    import torch
+    from paper_2304_01089_b200 import binding, calibration
+    from helpers import random_layout_params
+    rng = np.random.default_rng(21)
+    H, d, gh, T, C_in, g_in = 4, 64, 4, 130, 256, 6
+    perm1, size1, scale1, zero1 = random_layout_params(rng, C_in, g_in, 4)
+    L1 = binding.Layout(perm1, size1, scale1, zero1, 4)
+    a = codes_in_oracle_order(rng, T, size1, 4)
+    da = torch.from_numpy(oracle.pack(np.ascontiguousarray(a[:, L1.contiguous_position()]), 4)).cuda()
+    Ws = [(rng.normal(size=(H * d, C_in)) * 0.05 * rng.lognormal(0, 0.7, size=(H * d, 1))).astype(np.float32) for _ in range(3)]
+
+    def project(W, L_out):
+        n = H * d if L_out is None else L_out.K_pad
+        rows = None if L_out is None else L_out.padded_index().astype(np.int32)
+        w, s_w, wsum = binding.weight_pack(L1, W, out_perm=rows, n_pad=n)
+        dw, ds, dws = torch.from_numpy(w).cuda(), torch.from_numpy(s_w).cuda(), torch.from_numpy(wsum).cuda()
+        if L_out is None:
+            y = torch.empty((T, n), dtype=torch.float32, device="cuda")
+            binding.cluster_gemm(L1, da, T, dw, ds, dws, n, y)
+        else:
+            y = torch.empty((T, L_out.row_bytes), dtype=torch.uint8, device="cuda")
+            binding.cluster_gemm(L1, da, T, dw, ds, dws, n, y, layout_out=L_out, y_dtype=binding.OUT_CODES)
+        torch.cuda.synchronize()
+        return y
+
+    ranges = []
+    for W in Ws:                                   # calibration ranges from the projections' own outputs
+        y = project(W, None).cpu().numpy().astype(np.float64)
+        ranges.append((y.min(axis=0), y.max(axis=0)))
+    draws = rng.uniform(size=(H, gh))
+    cal_qk = calibration.calibrate_heads(ranges[:2], H, gh, (4, 4), draws, device="cuda")
+    cal_v = calibration.calibrate_heads(ranges[2:], H, gh, (3,), draws, device="cuda")
+    host_qk = calibration.calibrate_heads(ranges[:2], H, gh, (4, 4), draws)
+    assert np.array_equal(cal_qk.perm, host_qk.perm) and np.array_equal(cal_qk.size, host_qk.size)
+
+    c = Case.__new__(Case)
+    c.H, c.hd, c.gh, c.Tq, c.Tk = H, d, gh, T, T
+    c.perm_qk, c.size_qk, c.perm_v, c.size_v = cal_qk.perm, cal_qk.size, cal_v.perm, cal_v.size
+    (c.sQ, c.sK), (c.zQ, c.zK), c.sV, c.zV = cal_qk.scale, cal_qk.zero, cal_v.scale[0], cal_v.zero[0]
+    c.LQ = binding.Layout(c.perm_qk, c.size_qk, c.sQ, c.zQ, 4)
+    c.LK = binding.Layout(c.perm_qk, c.size_qk, c.sK, c.zK, 4)
+    c.LV = binding.Layout(c.perm_v, c.size_v, c.sV, c.zV, 3)
+    c.dq, c.dk, c.dv = project(Ws[0], c.LQ), project(Ws[1], c.LK), project(Ws[2], c.LV)
+    back = lambda t, L, b: oracle.unpack(t.cpu().numpy(), L.K_pad, b)[:, np.argsort(L.contiguous_position())]
+    c.q, c.k, c.v = back(c.dq, c.LQ, 4), back(c.dk, c.LK, 4), back(c.dv, c.LV, 3)
+    assert c.q.max() > 8 and c.k.max() > 8 and c.v.max() > 4          # the ranges are used
+    c.qk_scale, c.s_P = 1.0 / np.sqrt(d), 1.0 / 256
+    c.check(True)

@@ -209,3 +209,47 @@ def test_workload_generators_are_seeded_and_shaped():
     part = list(workloads.weight_rows(w, 0, 3072, 768, 1000, 1100))
     assert np.array_equal(np.concatenate([b for _, b in part]), full[1000:1100])
     assert abs(full.std() - 0.02) < 1e-3
+
+
+def _head_ranges(rng, H, d, planted):
+    """Per-channel (min, max) of Q and K with `planted` groups per head: the groups differ in K's range
+    only, so a clustering on Q's ranges alone cannot find them."""
+    group = np.concatenate([rng.permutation(np.arange(d) % planted) for _ in range(H)])
+    q_hi = rng.uniform(0.9, 1.1, size=H * d); q_lo = -rng.uniform(0.9, 1.1, size=H * d)
+    k_hi = (1.0 + 4.0 * group) * rng.uniform(0.95, 1.05, size=H * d); k_lo = -k_hi * rng.uniform(0.95, 1.05, size=H * d)
+    return (q_lo, q_hi), (k_lo, k_hi), group
+
+
+def test_attention_sites_share_one_index_between_q_and_k():
+    """Sec. 4.2: Q and K of a head are clustered together on (Q max, Q min, K max, K min); Sec. 5.1: per
+    head. The numpy calibration agrees with the oracle's composition, finds groups that only K's ranges
+    show, and gives each tensor its own Eq. 2 parameters on the shared clusters."""
+    rng = np.random.default_rng(3)
+    H, d, gh = 3, 32, 4
+    q, k, group = _head_ranges(rng, H, d, gh)
+    draws = rng.uniform(size=(H, gh))
+    cal = calibration.calibrate_heads([q, k], H, gh, (4, 3), draws)
+    perm, size, scale, zero = oracle.calibrate_heads([q, k], H, gh, (4, 3), draws)
+    assert np.array_equal(cal.perm, perm) and np.array_equal(cal.size, size)
+    for t in range(2):
+        assert np.array_equal(cal.scale[t], scale[t].astype(np.float32)) and np.array_equal(cal.zero[t], zero[t])
+    assert cal.size.shape == (H * gh,) and np.array_equal(np.sort(cal.perm), np.arange(H * d))
+    pos = 0
+    for h in range(H):
+        assert cal.size[h * gh:(h + 1) * gh].sum() == d
+        for c in range(gh):
+            n = int(cal.size[h * gh + c])
+            seg = cal.perm[pos:pos + n]
+            pos += n
+            assert np.all(seg // d == h)                        # a head's clusters hold that head's channels
+            assert len(set(group[seg])) == 1                    # and are the planted groups
+            for t, (lo, hi) in enumerate((q, k)):               # Eq. 2 on the cluster's merged range, per tensor
+                bits = (4, 3)[t]
+                s = (hi[seg].max() - lo[seg].min()) / (1 << bits)
+                assert cal.scale[t][h * gh + c] == np.float32(s)
+                assert cal.zero[t][h * gh + c] == -int(np.rint((hi[seg].max() + lo[seg].min()) / (2 * s))) + (1 << (bits - 1))
+    # a single tensor (R3, the values): the same routine with 2-D points
+    v = (k[0] * 0.5, k[1] * 0.5)
+    cv = calibration.calibrate_heads([v], H, gh, (4,), draws)
+    pv, sv, _, _ = oracle.calibrate_heads([v], H, gh, (4,), draws)
+    assert np.array_equal(cv.perm, pv) and np.array_equal(cv.size, sv)
