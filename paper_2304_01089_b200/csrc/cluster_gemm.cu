@@ -1092,6 +1092,16 @@ static int launch_gemm(const rptq_layout_t* Lin, const void* a_codes, int M, con
     int n_sm = 0;
     if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return RPTQ_ERR_CUDA;
     auto st = static_cast<cudaStream_t>(stream);
+    // a few tokens (decoding): the kernel that streams the weights through mma.sync with the channels as its M dimension
+    if (!deq && !sw_c && y_dtype != RPTQ_OUT_CODES && smallm::fits(M, Lin->bits, Lin->K_pad)) {
+        SmallMParams q{};
+        q.a = p.a_codes; q.a_row_bytes = p.a_row_bytes; q.M = M; q.K_pad = Lin->K_pad; q.n_units = Lin->n_units; q.n_kb = p.n_kb;
+        q.w = p.w_codes; q.n_wtiles = p.n_wtiles;
+        q.step_flags = Lin->d_step_flags; q.unit_cluster = Lin->d_unit_cluster; q.unit_sz = Lin->d_unit_sz; q.cl_sz = Lin->d_cl_sz; q.g = Lin->g;
+        q.corr = corr; q.s_w = s_w; q.wsum = wsum; q.ld_w = ld_w; q.bias = p.bias;
+        q.N = N; q.act = act; q.y_dtype = y_dtype; q.y = y; q.ldy = ldy; q.status = status;
+        return smallm::launch(q, Lin->bits, st);
+    }
     if (deq) {
         p.unit_sz = Lin->d_unit_sz;
         if (ncta == 2) {

@@ -56,6 +56,19 @@ struct rptq_layout {
 
 namespace rptq {
 
+// The cluster GEMM for at most 16 tokens (small_m_gemm.cu).
+struct SmallMParams {
+    const uint8_t* a; int64_t a_row_bytes; int M, K_pad, n_units, n_kb;
+    const uint8_t* w; int n_wtiles;
+    const uint8_t* step_flags; const int32_t* unit_cluster; const float2* unit_sz; const float* cl_sz; int g;
+    const float* corr; const float* s_w; const int32_t* wsum; int64_t ld_w; const float* bias;
+    int N, act, y_dtype; void* y; int64_t ldy; int* status;
+};
+namespace smallm {
+bool fits(int M, int bits, int K_pad);
+int launch(const SmallMParams& p, int bits, cudaStream_t st);
+}
+
 int* device_status_word();   // lazily allocated device int, RPTQ_OK when clear; nullptr on failure
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }

@@ -337,3 +337,30 @@ def test_workload_configs_checked_in_full(name):
     sub = slice(0, 8)
     ref = oracle.dequant_matmul(a[sub], w_codes, site.cal.size, site.cal.scale.astype(np.float64), site.cal.zero, s_w)
     assert np.max(np.abs(ref - want[sub])) <= 1e-10 * np.abs(want).max()
+
+
+@pytest.mark.parametrize("order", [0, 1])
+@pytest.mark.parametrize("bits", [4, 3, 8])
+def test_few_tokens_take_the_direct_kernel_and_give_the_same_bits(bits, order):
+    """Calls with at most 16 tokens run the kernel that feeds the weights straight into mma.sync (no
+    tensor-memory tile); its result is right against the oracle and bit-identical to what the large
+    kernel gives for the same tokens as part of a longer batch."""
+    from paper_2304_01089_b200 import binding
+    rng = np.random.default_rng(77 + bits + 10 * order)
+    M_all, N, C, g = 40, 300, 1024, 33
+    case = _case(rng, M_all, N, C, g, bits, n_pad=304)
+    d = _dev(case, order=order)
+    bias = (rng.normal(size=N) * 0.05).astype(np.float32)
+    want = _oracle_y(case, bias=bias, relu=True)
+    big = _gemm(case, d, bias=bias, act=binding.ACT_RELU, ldy=304)[:, :N]            # 40 tokens: the tcgen05 kernel
+    assert np.max(np.abs(big - want)) <= TOL * np.abs(want).max()
+    for M in (1, 7, 8, 9, 16):
+        sub = dict(case, M=M)
+        y32 = _gemm(sub, d, bias=bias, act=binding.ACT_RELU, ldy=304)[:, :N]
+        assert np.max(np.abs(y32 - want[:M])) <= TOL * np.abs(want).max()
+        assert np.array_equal(y32, big[:M])
+        y16 = _gemm(sub, d, y_dtype=binding.OUT_F16, bias=bias, act=binding.ACT_RELU, ldy=304)[:, :N]
+        assert np.array_equal(y16, big[:M].astype(np.float16))
+    # no bias, no activation, an output pitch wider than N
+    y = _gemm(dict(case, M=5), d, ldy=320)[:, :N]
+    assert np.max(np.abs(y - _oracle_y(case)[:5])) <= TOL * np.abs(want).max()
