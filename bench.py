@@ -132,6 +132,43 @@ def _step(sites, binding, M, events=None):
             events[i][2].record()
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one FC1 launch, from the 512-token ncu capture of the
+# current kernel (profiles/cluster_gemm_opt66b_fc1_tokens512.txt: 191.5 MB read, 23.4 MB written, part of
+# the output still in L2) scaled to 4096 tokens: weights, Wsum and s_w (191.1 MB) are read once whatever
+# the token count; codes (1.94 MB per 512 tokens) and the fp16 output (37.75 MB per 512 tokens) grow with it.
+FC1_DRAM_BYTES_PER_LAUNCH = int(191.1e6 + 8 * (1.94e6 + 37.75e6))
+
+
+def _attention_leg(w, M, torch, binding):
+    """rptq_attention at the workload's head shape (hidden / 128 heads of 128 channels, four clusters per
+    head, causal, one sequence of min(tokens, 2048)), on seeded codes. Not part of the timed step."""
+    from paper_2304_01089_b200 import workloads
+    site = workloads.attention_site(w)
+    H, T = site["heads"], min(M, 2048)
+    LQ = binding.Layout(site["perm_qk"], site["size_qk"], site["scale"]["q"], site["zero"]["q"], w.bits)
+    LK = binding.Layout(site["perm_qk"], site["size_qk"], site["scale"]["k"], site["zero"]["k"], w.bits)
+    LV = binding.Layout(site["perm_v"], site["size_v"], site["scale"]["v"], site["zero"]["v"], w.bits)
+    dev = [torch.from_numpy(binding.codes_pack_host(workloads.attention_codes(w, T, L.padded_index() >= 0, t), w.bits)).cuda()
+           for t, L in enumerate((LQ, LK, LV))]
+    out = torch.empty((T, w.hidden), dtype=torch.float16, device="cuda")
+    run = lambda: binding.attention(LQ, LK, LV, H, dev[0], dev[1], dev[2], out, 1.0 / 256, 1.0 / np.sqrt(128.0), True)
+    for _ in range(3):
+        run()
+    n_rep = 10
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(n_rep + 1)]
+    torch.cuda.synchronize()
+    for i in range(n_rep):
+        ev[i].record()
+        run()
+    ev[n_rep].record()
+    torch.cuda.synchronize()
+    us = float(np.median([ev[i].elapsed_time(ev[i + 1]) for i in range(n_rep)])) * 1e3
+    ops = 2.0 * H * (T * (T + 1) / 2) * 128 * 2            # both products once, visible keys, real channels
+    return {"kernel": "attention_kernel", "heads": H, "head_dim": 128, "clusters_per_head": 4, "tokens": T, "causal": True,
+            "bits": w.bits, "us": us, "TOPS": ops / us / 1e6,
+            "note": "integer products on mma.sync m16n8k32 (the scores are computed twice: the softmax codes need the finished row sums)"}
+
+
 def run_ours(args):
     import torch
     from paper_2304_01089_b200 import binding, shard, workloads
@@ -228,6 +265,7 @@ def run_ours(args):
             sweep.append({"kernel": "cluster_gemm FC1", "tokens": m_small, "us": us,
                           "TOPS": 2.0 * m_small * C * fc["n_out"] / us / 1e6,
                           "weight_stream_GBps": w_bytes / us / 1e3, "weight_bytes": w_bytes})
+        attention = _attention_leg(w, M, torch, binding)
         failed = torch.zeros(1, dtype=torch.int32, device="cuda")
         binding.probe_int8_peak(200, failed)
         p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -279,7 +317,7 @@ def run_ours(args):
                 "cluster_gemm_fc1": {"ms": fc1_ms, "TOPS": achieved},
             },
             "roofline": {"bound": "tensor", "achieved": achieved, "peak": proxy, "unit": "TOP/s",
-                         "frac": achieved / proxy, "traffic": None,
+                         "frac": achieved / proxy, "traffic": FC1_DRAM_BYTES_PER_LAUNCH if M == 4096 else None,
                          "kernel": "cluster_gemm_kernel<3> 4096x9216x36864",
                          "peak_note": (f"2 x bf16 {'burst' if at_max_clock else 'sustained'} of {peaks['source']} peaks: a proxy "
                                        "(nominal int8 : bf16 ratio), not an int8 measurement; the own-dtype ceiling is peak_int8_measured"),
@@ -293,6 +331,7 @@ def run_ours(args):
                    "frac": ln_gbs / peaks["hbm"], "frac_of_8TBps": ln_gbs / 8000.0, "bytes": ln_bytes,
                    "us": float(np.mean(ln_ms[1])) * 1e3},
             "sweep": sweep,
+            "attention": attention,
             "e2e": None if args.no_e2e else {"value": world * ops_per_step * e2e_steps / (e2e_ms * 1e-3) / 1e12, "unit": "TOPS",
                     "h2d_bytes_per_step": int(sum(s["x_host"].numel() * 2 for s in sites)),
                     "d2h_bytes_per_step": int(sum(s["y_host"].numel() * 2 for s in sites))},

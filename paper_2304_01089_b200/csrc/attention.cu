@@ -15,7 +15,8 @@
 // (P_q's zero point is required to be 0). The scores' 16 x 8 accumulator blocks give each thread two
 // adjacent keys of a row; four of them (from two blocks) form one operand word of the second product,
 // so the keys of a tile enter that product in a permuted order, and the V tile is transposed into
-// shared memory in the same order. Pass 2 runs once per chunk of four V units (128 positions).
+// shared memory in the same order. Pass 2 holds the sums of up to eight V units (a whole head) in
+// registers; a head with more units would take another sweep over the keys per eight units.
 #include <cuda_fp16.h>
 
 #include "rptq_internal.h"
@@ -27,7 +28,7 @@ namespace attn {
 constexpr int BM = 64, BN = 64, THREADS = 128;
 constexpr int MAX_UNITS = 8;                 // units of 32 positions per head
 constexpr int QK_PITCH_MAX = 32 * MAX_UNITS + 16;
-constexpr int V_CHUNK_UNITS = 4;
+constexpr int V_CHUNK_UNITS = 8;
 constexpr int VT_PITCH = BN + 16;
 constexpr float NEG_BIG = -1.0e30f;
 

@@ -55,7 +55,7 @@ WORKLOADS: Dict[str, Workload] = {
 }
 
 # stream tags keep the different tensors of one workload statistically independent
-_TAG_LN, _TAG_TEST, _TAG_CALIB, _TAG_W, _TAG_KMEANS, _TAG_BIAS = 11, 12, 13, 14, 15, 16
+_TAG_LN, _TAG_TEST, _TAG_CALIB, _TAG_W, _TAG_KMEANS, _TAG_BIAS, _TAG_HEADS = 11, 12, 13, 14, 15, 16, 17
 
 
 def _rng(seed: int, tag: int, *extra: int) -> np.random.Generator:
@@ -152,3 +152,34 @@ def kmeans_draws(w: Workload, site: int, g: int) -> np.ndarray:
     here and handed to whichever clustering code runs, so two implementations that follow the
     same steps pick the same seeds."""
     return _rng(w.seed, _TAG_KMEANS, site).random(g)
+
+
+def attention_site(w: Workload, head_dim: int = 128, clusters_per_head: int = 4):
+    """Seeded stand-in for the calibrated attention sites of the workload's model (reorders R2 / R3 of the
+    paper, computed per head with four clusters): per head a random permutation of its channels, cluster
+    sizes drawn around head_dim / clusters_per_head, and per-cluster scales and zero points for Q, K and
+    V. Returns dict(heads, perm_qk, size_qk, perm_v, size_v, scale={q,k,v}, zero={q,k,v}); Q and K share
+    perm_qk / size_qk. Code tensors come from attention_codes."""
+    r = _rng(w.seed, _TAG_HEADS)
+    heads = w.hidden // head_dim
+    def index():
+        perm, size = [], []
+        for h in range(heads):
+            perm.append(h * head_dim + r.permutation(head_dim))
+            size.append(1 + r.multinomial(head_dim - clusters_per_head, np.ones(clusters_per_head) / clusters_per_head))
+        return np.concatenate(perm).astype(np.int32), np.concatenate(size).astype(np.int32)
+    perm_qk, size_qk = index()
+    perm_v, size_v = index()
+    g = heads * clusters_per_head
+    scale = {t: r.uniform(0.05, 0.3, size=g).astype(np.float32) for t in "qkv"}
+    zero = {t: r.integers(0, 1 << w.bits, size=g).astype(np.int32) for t in "qkv"}
+    return dict(heads=heads, perm_qk=perm_qk, size_qk=size_qk, perm_v=perm_v, size_v=size_v, scale=scale, zero=zero)
+
+
+def attention_codes(w: Workload, tokens: int, real_position: np.ndarray, tensor: int) -> np.ndarray:
+    """uint8 [tokens][K_pad] uniform codes of w.bits bits at the real positions of a layout (real_position:
+    bool [K_pad]), zero at its pad positions. tensor: 0, 1, 2 for Q, K, V."""
+    r = _rng(w.seed, _TAG_HEADS, 1 + tensor)
+    codes = r.integers(0, 1 << w.bits, size=(tokens, real_position.shape[0]), dtype=np.uint8)
+    codes[:, ~real_position] = 0
+    return codes
