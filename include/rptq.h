@@ -2,11 +2,15 @@
  * rptq.h -- C boundary of the B200 (sm_100a) library for the hot path of RPTQ, reorder-based
  * post-training quantisation (arXiv 2304.01089).
  *
- * The library holds two device kernels and the small amount of host logic around them:
+ * The two calls of the hot path, and the small amount of host logic around them:
  *
  *   rptq_ln_reorder_quant   LayerNorm -> channel reorder -> per-cluster quantise -> packed codes
  *   rptq_cluster_gemm       packed activation codes x packed int4 weights, integer products per
- *                           cluster segment on the tensor cores, floating-point epilogue
+ *                           cluster segment on the tensor cores, floating-point epilogue (calls
+ *                           with at most 16 tokens run a second kernel with the same arithmetic)
+ * Further down: the same product with per-cluster asymmetric weights or as a de-quantised
+ * bfloat16 product, attention on quantised Q / K / V, calibration on the device, and aids for
+ * tests and measurement.
  *
  * Conventions
  *   - Every function returns an int status: RPTQ_OK or a negative RPTQ_ERR_* value. Nothing
