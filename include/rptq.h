@@ -203,8 +203,8 @@ int rptq_dequant_gemm(const rptq_layout_t* Lin, const void* a_codes, int M, cons
                       void* y, int y_dtype, int64_t ldy, void* stream);
 
 /*
- * Appendix: "for one output channel, each weight cluster is quantised with its own asymmetric
- * parameters", W~_q,i = Q_k(W~_i, s^W_i, z^W_i), the paper's own weight scheme (it finds the codes
+ * Appendix: the weights of an output channel get one asymmetric (scale, zero point) pair per input
+ * cluster, W~_q,i = Q_k(W~_i, s^W_i, z^W_i), the paper's own weight scheme (it finds the codes
  * with GPTQ; here round-to-nearest). For output row r and input cluster c with n_c > 0, in fp32:
  *   s = (max - min) / 16 over the row's weights of the cluster (1 if max == min)       [Eq. 2, k = 4]
  *   z = 8 - rne((max + min) / (2 s)),   W_q = clamp(rne(W / s) + z, 0, 15)           [Eq. 1, re-based]

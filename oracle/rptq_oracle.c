@@ -572,8 +572,8 @@ void orc_dequant_matmul(const uint8_t* a_codes, int64_t M, const int8_t* w_codes
 /* Per-cluster asymmetric weight parameters (Appendix, W~_q,i = Q_k(W~_i, s^W_i, z^W_i))       */
 /* ------------------------------------------------------------------------------------------ */
 
-/* Appendix: "for one output channel, each weight cluster is quantised with its own asymmetric
- * parameters". For output row r and input cluster i the parameters come from the Min-Max method
+/* Appendix: the weights of an output channel get one asymmetric (scale, zero point) pair per input
+ * cluster. For output row r and input cluster i the parameters come from the Min-Max method
  * (Eq. 2, taken literally as for the activations) over the row's weights of that cluster, and the
  * codes from Eq. 1 re-based to [0, 2^k - 1]. (The paper obtains the codes with GPTQ, which needs a
  * trained model's Hessians; round-to-nearest is used here.) Everything that decides an integer is
