@@ -358,7 +358,7 @@ int rptq_selftest_ln_timeout(const rptq_layout_t* L, const void* x, int64_t ldx,
  * Layouts: LQ, LK, LV have n_heads * (clusters per head) clusters in RPTQ_ORDER_CONTIGUOUS order, head h
  * owning clusters h * g / n_heads .. (h + 1) * g / n_heads - 1 and the channels h * d .. (h + 1) * d - 1;
  * LQ and LK must have the same reorder index and cluster sizes (their scales and zero points differ).
- * A head may take at most 8 units of 32 positions in LQ / LK.
+ * A head may take at most 8 units of 32 positions in each layout.
  *   q_codes  dev, Tq rows of LQ.row_bytes bytes (as an RPTQ_OUT_CODES GEMM writes them)
  *   k_codes, v_codes  dev, Tk rows of LK.row_bytes / LV.row_bytes bytes: the quantised key / value cache
  *   s_P, z_P Eq. 1 parameters of the softmax output for codes in [0, 255]; z_P must be 0 (Eq. 2 on a

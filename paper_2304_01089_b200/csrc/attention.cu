@@ -16,7 +16,8 @@
 // adjacent keys of a row; four of them (from two blocks) form one operand word of the second product,
 // so the keys of a tile enter that product in a permuted order, and the V tile is transposed into
 // shared memory in the same order. Pass 2 holds the sums of up to eight V units (a whole head) in
-// registers; a head with more units would take another sweep over the keys per eight units.
+// registers. The packed codes of the next key tile are copied into a staging buffer (cp.async) while
+// the current tile is multiplied.
 #include <cuda_fp16.h>
 
 #include "rptq_internal.h"
@@ -46,6 +47,7 @@ struct Params {
     __half* out;
     int64_t ldo;
     uint8_t* p_dbg;
+    int raw_pitch;                           // bytes per key row of the staging buffers for packed codes
 };
 
 __device__ __forceinline__ void load_unit(const uint8_t* row, int unit, int bits, uint32_t (&o)[8])
@@ -66,6 +68,32 @@ __device__ __forceinline__ void load_unit(const uint8_t* row, int unit, int bits
 }
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+// The same from a staged copy of the packed row in shared memory (`row` points at the head's first unit;
+// 4-byte aligned for 3-bit codes, 16-byte aligned otherwise).
+__device__ __forceinline__ void load_unit_smem(const uint8_t* row, int unit, int bits, uint32_t (&o)[8])
+{
+    if (bits == 4) {
+        const uint4 t = *(reinterpret_cast<const uint4*>(row) + unit);
+        const uint32_t p[4] = {t.x, t.y, t.z, t.w};
+        unpack_act32<4>(p, o);
+    } else if (bits == 3) {
+        const uint32_t* w = reinterpret_cast<const uint32_t*>(row) + unit * 3;
+        const uint32_t p[3] = {w[0], w[1], w[2]};
+        unpack_act32<3>(p, o);
+    } else {
+        const uint4* w = reinterpret_cast<const uint4*>(row) + unit * 2;
+        const uint4 a = w[0], b = w[1];
+        o[0] = a.x; o[1] = a.y; o[2] = a.z; o[3] = a.w; o[4] = b.x; o[5] = b.y; o[6] = b.z; o[7] = b.w;
+    }
+}
+// 16 bytes global -> shared without passing through registers; src_bytes = 0 writes zeros
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int src_bytes)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 __device__ __forceinline__ void ldsm4(uint32_t addr, uint32_t (&r)[4])
 {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
@@ -128,6 +156,12 @@ attention_kernel(const Params p)
     uint8_t* Qs = smem;
     uint8_t* Ks = Qs + BM * QK_PITCH_MAX;
     uint8_t* Vt = Ks + BN * QK_PITCH_MAX;
+    uint8_t* rawK = Vt + 32 * V_CHUNK_UNITS * VT_PITCH;         // [2][BN][raw_pitch] packed K codes of a tile, as they lie in memory
+    uint8_t* rawV = rawK + 2 * BN * p.raw_pitch;
+    // a head's packed codes are a contiguous piece of a row; the staged window starts at the 16-byte boundary below it
+    const int bytesK = 4 * p.bits_k, bytesV = 4 * p.bits_v;
+    const int winK = (bytesK * uq0) & ~15, offK = bytesK * uq0 - winK, nK16 = (offK + bytesK * nuq + 15) >> 4;
+    const int winV = (bytesV * uv0) & ~15, offV = bytesV * uv0 - winV, nV16 = (offV + bytesV * nuv + 15) >> 4;
 
     if (tid < nuq) {
         const float2 q = __ldg(p.unit_sz_q + uq0 + tid), k = __ldg(p.unit_sz_k + uq0 + tid);
@@ -154,11 +188,29 @@ attention_kernel(const Params p)
     const int vis0 = p.causal ? min(p.Tk - 1, row0 + off) : p.Tk - 1;
     const int vis1 = p.causal ? min(p.Tk - 1, row1 + off) : p.Tk - 1;
 
+    // Start the copies of key tile kt (and its V tile) into staging buffer kt & 1; rows past the last key are zero-filled.
+    auto stage_tile = [&](int kt, bool with_v) {
+        const int buf = kt & 1;
+        for (int it = tid; it < BN * nK16; it += THREADS) {
+            const int r = it / nK16, c = it - r * nK16, j = kt * BN + r;
+            cp_async16(smem_u32(rawK + (buf * BN + r) * p.raw_pitch + 16 * c),
+                       p.k + (int64_t)min(j, p.Tk - 1) * p.k_row_bytes + winK + 16 * c, j < p.Tk ? 16 : 0);
+        }
+        if (with_v)
+            for (int it = tid; it < BN * nV16; it += THREADS) {
+                const int r = it / nV16, c = it - r * nV16, j = kt * BN + r;
+                cp_async16(smem_u32(rawV + (buf * BN + r) * p.raw_pitch + 16 * c),
+                           p.v + (int64_t)min(j, p.Tk - 1) * p.v_row_bytes + winV + 16 * c, j < p.Tk ? 16 : 0);
+            }
+        cp_async_commit();
+    };
+    // Tile kt has been staged and a block-wide barrier passed since: unpack it to bytes
     auto load_k_tile = [&](int kt) {
+        const uint8_t* raw = rawK + (kt & 1) * BN * p.raw_pitch + offK;
         for (int it = tid; it < BN * nuq; it += THREADS) {
             const int r = it / nuq, u = it - r * nuq;
-            uint32_t o[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-            if (kt * BN + r < p.Tk) load_unit(p.k + (int64_t)(kt * BN + r) * p.k_row_bytes, uq0 + u, p.bits_k, o);
+            uint32_t o[8];
+            load_unit_smem(raw + r * p.raw_pitch, u, p.bits_k, o);
             uint4* d = reinterpret_cast<uint4*>(Ks + r * pitch + 32 * u);
             d[0] = make_uint4(o[0], o[1], o[2], o[3]);
             d[1] = make_uint4(o[4], o[5], o[6], o[7]);
@@ -220,7 +272,10 @@ attention_kernel(const Params p)
 
     // ---------------------------------------------------------------- pass 1: row maximum and row sum
     float m0 = NEG_BIG, m1 = NEG_BIG, l0 = 0.f, l1 = 0.f;
+    stage_tile(0, false);
     for (int kt = 0; kt < n_kt; ++kt) {
+        if (kt + 1 < n_kt) { stage_tile(kt + 1, false); cp_async_wait<1>(); } else cp_async_wait<0>();
+        __syncthreads();                     // everyone's copies of tile kt have landed
         load_k_tile(kt);
         float S[8][4];
         scores(kt, S);
@@ -257,19 +312,19 @@ attention_kernel(const Params p)
 #pragma unroll
             for (int e = 0; e < 4; ++e) O[n][e] = 0;
         int rs0 = 0, rs1 = 0;                // sums of my rows' codes (this thread's keys)
+        stage_tile(0, true);
         for (int kt = 0; kt < n_kt; ++kt) {
+            if (kt + 1 < n_kt) { stage_tile(kt + 1, true); cp_async_wait<1>(); } else cp_async_wait<0>();
+            __syncthreads();                 // everyone's copies of tile kt have landed
             load_k_tile(kt);
             // V tile, transposed: Vt[position][slot] = code of key key_of_slot(slot)
+            const uint8_t* rawv = rawV + (kt & 1) * BN * p.raw_pitch + offV;
             for (int it = tid; it < cu * 16; it += THREADS) {
                 const int u = it >> 4, w = it & 15;
                 uint32_t o[4][8];
 #pragma unroll
-                for (int b = 0; b < 4; ++b) {
-                    const int j = kt * BN + key_of_slot(4 * w + b);
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) o[b][e] = 0;
-                    if (j < p.Tk) load_unit(p.v + (int64_t)j * p.v_row_bytes, uv0 + c0 + u, p.bits_v, o[b]);
-                }
+                for (int b = 0; b < 4; ++b)
+                    load_unit_smem(rawv + key_of_slot(4 * w + b) * p.raw_pitch, c0 + u, p.bits_v, o[b]);
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {        // positions 4e..4e+3 of the unit: a 4 x 4 byte transpose
                     const uint32_t x01l = __byte_perm(o[0][e], o[1][e], 0x5140), x01h = __byte_perm(o[0][e], o[1][e], 0x7362);
@@ -388,7 +443,7 @@ extern "C" int rptq_attention(const rptq_layout_t* LQ, const rptq_layout_t* LK, 
     if (z_P != 0) return RPTQ_ERR_UNSUPPORTED;
     int n_used_qk = 0, n_used_v = 0;
     if (!units_in_cluster_order(LQ, &n_used_qk) || !units_in_cluster_order(LV, &n_used_v)) return RPTQ_ERR_UNSUPPORTED;
-    if (max_units_per_head(LQ, n_used_qk, n_heads) > MAX_UNITS || max_units_per_head(LV, n_used_v, n_heads) > 255) return RPTQ_ERR_UNSUPPORTED;
+    if (max_units_per_head(LQ, n_used_qk, n_heads) > MAX_UNITS || max_units_per_head(LV, n_used_v, n_heads) > MAX_UNITS) return RPTQ_ERR_UNSUPPORTED;
     if ((int64_t)Tk * 255 * 255 > 2147483647ll) return RPTQ_ERR_UNSUPPORTED;      // the int32 sums of the second product
     if (Tq == 0) return RPTQ_OK;
     int dev = -1;
@@ -407,7 +462,9 @@ extern "C" int rptq_attention(const rptq_layout_t* LQ, const rptq_layout_t* LK, 
     p.inv_sP = 1.0f / s_P; p.s_P = s_P; p.qk_scale_log2e = qk_scale * 1.4426950408889634f;
     p.out = static_cast<__half*>(out_f16); p.ldo = ldo; p.p_dbg = p_codes_out;
 
-    const int smem = (BM + BN) * QK_PITCH_MAX + 32 * V_CHUNK_UNITS * VT_PITCH;
+    const int max_bits = LK->bits > LV->bits ? LK->bits : LV->bits;
+    p.raw_pitch = 4 * max_bits * MAX_UNITS + 32;          // a head's packed codes plus the alignment slack, a multiple of 16
+    const int smem = (BM + BN) * QK_PITCH_MAX + 32 * V_CHUNK_UNITS * VT_PITCH + 4 * BN * p.raw_pitch;
     if (cudaFuncSetAttribute(attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return RPTQ_ERR_CUDA;
     const dim3 grid((unsigned)((Tq + BM - 1) / BM), (unsigned)n_heads);
     if (n_heads > 65535) return RPTQ_ERR_UNSUPPORTED;
