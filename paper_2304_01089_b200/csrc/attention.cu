@@ -440,7 +440,7 @@ extern "C" int rptq_attention(const rptq_layout_t* LQ, const rptq_layout_t* LK, 
     // Q and K pair equal positions: same reorder index, same cluster sizes, same placement
     if (LQ->C != LK->C || LQ->size != LK->size || LQ->perm != LK->perm || LQ->pos != LK->pos || LQ->unit_cluster != LK->unit_cluster)
         return RPTQ_ERR_INVALID_ARG;
-    if (z_P != 0) return RPTQ_ERR_UNSUPPORTED;
+    if (z_P != 0 || n_heads > 65535) return RPTQ_ERR_UNSUPPORTED;
     int n_used_qk = 0, n_used_v = 0;
     if (!units_in_cluster_order(LQ, &n_used_qk) || !units_in_cluster_order(LV, &n_used_v)) return RPTQ_ERR_UNSUPPORTED;
     if (max_units_per_head(LQ, n_used_qk, n_heads) > MAX_UNITS || max_units_per_head(LV, n_used_v, n_heads) > MAX_UNITS) return RPTQ_ERR_UNSUPPORTED;
@@ -467,7 +467,6 @@ extern "C" int rptq_attention(const rptq_layout_t* LQ, const rptq_layout_t* LK, 
     const int smem = (BM + BN) * QK_PITCH_MAX + 32 * V_CHUNK_UNITS * VT_PITCH + 4 * BN * p.raw_pitch;
     if (cudaFuncSetAttribute(attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return RPTQ_ERR_CUDA;
     const dim3 grid((unsigned)((Tq + BM - 1) / BM), (unsigned)n_heads);
-    if (n_heads > 65535) return RPTQ_ERR_UNSUPPORTED;
     attention_kernel<<<grid, THREADS, smem, static_cast<cudaStream_t>(stream)>>>(p);
     return cudaGetLastError() == cudaSuccess ? RPTQ_OK : RPTQ_ERR_CUDA;
 }
