@@ -141,17 +141,18 @@ FC1_DRAM_BYTES_PER_LAUNCH = int(191.1e6 + 8 * (1.94e6 + 37.75e6))
 
 def _attention_leg(w, M, torch, binding):
     """rptq_attention at the workload's head shape (hidden / 128 heads of 128 channels, four clusters per
-    head, causal, one sequence of min(tokens, 2048)), on seeded codes. Not part of the timed step."""
+    head, causal, tokens / 2048 sequences of 2048 tokens (one shorter sequence below that), on seeded codes. Not part of the timed step."""
     from paper_2304_01089_b200 import workloads
     site = workloads.attention_site(w)
     H, T = site["heads"], min(M, 2048)
+    n_seq = max(1, M // T)                                 # 4096 tokens: two sequences of 2048 in one call
     LQ = binding.Layout(site["perm_qk"], site["size_qk"], site["scale"]["q"], site["zero"]["q"], w.bits)
     LK = binding.Layout(site["perm_qk"], site["size_qk"], site["scale"]["k"], site["zero"]["k"], w.bits)
     LV = binding.Layout(site["perm_v"], site["size_v"], site["scale"]["v"], site["zero"]["v"], w.bits)
-    dev = [torch.from_numpy(binding.codes_pack_host(workloads.attention_codes(w, T, L.padded_index() >= 0, t), w.bits)).cuda()
+    dev = [torch.from_numpy(binding.codes_pack_host(workloads.attention_codes(w, n_seq * T, L.padded_index() >= 0, t), w.bits)).cuda()
            for t, L in enumerate((LQ, LK, LV))]
-    out = torch.empty((T, w.hidden), dtype=torch.float16, device="cuda")
-    run = lambda: binding.attention(LQ, LK, LV, H, dev[0], dev[1], dev[2], out, 1.0 / 256, 1.0 / np.sqrt(128.0), True)
+    out = torch.empty((n_seq * T, w.hidden), dtype=torch.float16, device="cuda")
+    run = lambda: binding.attention(LQ, LK, LV, H, dev[0], dev[1], dev[2], out, 1.0 / 256, 1.0 / np.sqrt(128.0), True, n_seq=n_seq)
     for _ in range(3):
         run()
     n_rep = 10
@@ -163,8 +164,8 @@ def _attention_leg(w, M, torch, binding):
     ev[n_rep].record()
     torch.cuda.synchronize()
     us = float(np.median([ev[i].elapsed_time(ev[i + 1]) for i in range(n_rep)])) * 1e3
-    ops = 2.0 * H * (T * (T + 1) / 2) * 128 * 2            # both products once, visible keys, real channels
-    return {"kernel": "attention_kernel", "heads": H, "head_dim": 128, "clusters_per_head": 4, "tokens": T, "causal": True,
+    ops = 2.0 * n_seq * H * (T * (T + 1) / 2) * 128 * 2    # both products once, visible keys, real channels
+    return {"kernel": "attention_kernel", "heads": H, "head_dim": 128, "clusters_per_head": 4, "sequences": n_seq, "tokens": T, "causal": True,
             "bits": w.bits, "us": us, "TOPS": ops / us / 1e6,
             "note": "integer products on mma.sync m16n8k32 (the scores are computed twice: the softmax codes need the finished row sums)"}
 

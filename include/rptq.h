@@ -359,17 +359,18 @@ int rptq_selftest_ln_timeout(const rptq_layout_t* L, const void* x, int64_t ldx,
  * owning clusters h * g / n_heads .. (h + 1) * g / n_heads - 1 and the channels h * d .. (h + 1) * d - 1;
  * LQ and LK must have the same reorder index and cluster sizes (their scales and zero points differ).
  * A head may take at most 8 units of 32 positions in each layout.
- *   q_codes  dev, Tq rows of LQ.row_bytes bytes (as an RPTQ_OUT_CODES GEMM writes them)
- *   k_codes, v_codes  dev, Tk rows of LK.row_bytes / LV.row_bytes bytes: the quantised key / value cache
+ *   n_seq    sequences in the call, each with Tq queries and Tk keys; their rows follow one another
+ *   q_codes  dev, n_seq * Tq rows of LQ.row_bytes bytes (as an RPTQ_OUT_CODES GEMM writes them)
+ *   k_codes, v_codes  dev, n_seq * Tk rows of LK.row_bytes / LV.row_bytes bytes: the quantised key / value cache
  *   s_P, z_P Eq. 1 parameters of the softmax output for codes in [0, 255]; z_P must be 0 (Eq. 2 on a
  *            range that starts at 0 gives exactly that), otherwise RPTQ_ERR_UNSUPPORTED
- *   out_f16  dev fp16 [Tq][ldo], ldo >= LV.C: channel ch of token i at out[i * ldo + ch]
- *   p_codes_out  NULL, or dev uint8 [n_heads][Tq][Tk]: receives P_q at the visible keys of key tiles
+ *   out_f16  dev fp16 [n_seq * Tq][ldo], ldo >= LV.C: channel ch of query row i at out[i * ldo + ch]
+ *   p_codes_out  NULL, or dev uint8 [n_seq][n_heads][Tq][Tk]: receives P_q at the visible keys of key tiles
  *            that hold a visible key (a test aid; clear it before the call)
- * Tk >= Tq; Tk * 255 * 255 < 2^31. Row-constant terms of A cancel in the softmax and are not formed.
+ * Tk >= Tq; Tk * 255 * 255 < 2^31; n_seq, n_heads <= 65535. Row-constant terms of A cancel in the softmax and are not formed.
  */
 int rptq_attention(const rptq_layout_t* LQ, const rptq_layout_t* LK, const rptq_layout_t* LV, int n_heads,
-                   const void* q_codes, int Tq, const void* k_codes, const void* v_codes, int Tk,
+                   const void* q_codes, int Tq, const void* k_codes, const void* v_codes, int Tk, int n_seq,
                    float s_P, int z_P, float qk_scale, int causal,
                    void* out_f16, int64_t ldo, uint8_t* p_codes_out, void* stream);
 

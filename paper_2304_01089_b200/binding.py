@@ -70,7 +70,7 @@ def _load(path: str = LIB_PATH) -> C.CDLL:
     lib.rptq_get_device_status.argtypes = [C.POINTER(i32)]
     lib.rptq_status_string.argtypes = [i32]
     lib.rptq_status_string.restype = C.c_char_p
-    lib.rptq_attention.argtypes = [vp, vp, vp, i32, vp, i32, vp, vp, i32, f32, i32, f32, i32, vp, i64, vp, vp]
+    lib.rptq_attention.argtypes = [vp, vp, vp, i32, vp, i32, vp, vp, i32, i32, f32, i32, f32, i32, vp, i64, vp, vp]
     for name in EXPORTS:
         if name not in ("rptq_status_string", "rptq_weight_codes_bytes", "rptq_kmeans_workspace_bytes"):
             getattr(lib, name).restype = i32
@@ -209,13 +209,14 @@ def selftest_ln_timeout(layout: Layout, x, gamma, beta, eps: float, codes, M: Op
 
 def attention(LQ: Layout, LK: Layout, LV: Layout, n_heads: int, q_codes, k_codes, v_codes, out, s_P: float,
               qk_scale: float, causal: bool, z_P: int = 0, Tq: Optional[int] = None, Tk: Optional[int] = None,
-              p_codes=None, stream=None) -> None:
-    """rptq_attention: q_codes uint8 [Tq][LQ.row_bytes], k_codes / v_codes uint8 [Tk][row_bytes] CUDA tensors,
-    out fp16 [Tq][>= LV.C]; p_codes: optional uint8 [n_heads][Tq][Tk] (zeroed by the caller)."""
-    Tq = int(q_codes.shape[0]) if Tq is None else int(Tq)
-    Tk = int(k_codes.shape[0]) if Tk is None else int(Tk)
+              n_seq: int = 1, p_codes=None, stream=None) -> None:
+    """rptq_attention on n_seq sequences of Tq queries and Tk keys each: q_codes uint8 [n_seq * Tq][LQ.row_bytes],
+    k_codes / v_codes uint8 [n_seq * Tk][row_bytes] CUDA tensors, out fp16 [n_seq * Tq][>= LV.C]; p_codes:
+    optional uint8 [n_seq][n_heads][Tq][Tk] (zeroed by the caller)."""
+    Tq = int(q_codes.shape[0]) // int(n_seq) if Tq is None else int(Tq)
+    Tk = int(k_codes.shape[0]) // int(n_seq) if Tk is None else int(Tk)
     _check(_lib.rptq_attention(LQ.handle, LK.handle, LV.handle, int(n_heads), _dev_ptr(q_codes), Tq, _dev_ptr(k_codes),
-                               _dev_ptr(v_codes), Tk, C.c_float(s_P), int(z_P), C.c_float(qk_scale), 1 if causal else 0,
+                               _dev_ptr(v_codes), Tk, int(n_seq), C.c_float(s_P), int(z_P), C.c_float(qk_scale), 1 if causal else 0,
                                _dev_ptr(out), int(out.stride(0)), _dev_ptr(p_codes), _stream_ptr(stream)), "rptq_attention")
 
 

@@ -37,7 +37,7 @@ struct Params {
     const uint8_t *q, *k, *v;
     int64_t q_row_bytes, k_row_bytes, v_row_bytes;
     int bits_q, bits_k, bits_v;
-    int Tq, Tk, H, gh_qk, gh_v, causal;
+    int Tq, Tk, H, gh_qk, gh_v, causal;     // Tq queries and Tk keys per sequence; blockIdx.z is the sequence
     int n_used_qk, n_used_v;                 // units that belong to a cluster
     const int32_t *unit_cluster_qk, *unit_cluster_v;
     const float2 *unit_sz_q, *unit_sz_k, *unit_sz_v;
@@ -141,6 +141,7 @@ attention_kernel(const Params p)
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g8 = lane >> 2, t4 = lane & 3;
     const int h = blockIdx.y;
+    const int64_t q_row0 = (int64_t)blockIdx.z * p.Tq, k_row0 = (int64_t)blockIdx.z * p.Tk;      // this sequence's first rows
     const int qt = (int)gridDim.x - 1 - (int)blockIdx.x;      // the tiles with the most visible keys first
     const int i0 = qt * BM;
 
@@ -174,7 +175,7 @@ attention_kernel(const Params p)
     for (int it = tid; it < BM * nuq; it += THREADS) {
         const int r = it / nuq, u = it - r * nuq;
         uint32_t o[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-        if (i0 + r < p.Tq) load_unit(p.q + (int64_t)(i0 + r) * p.q_row_bytes, uq0 + u, p.bits_q, o);
+        if (i0 + r < p.Tq) load_unit(p.q + (q_row0 + i0 + r) * p.q_row_bytes, uq0 + u, p.bits_q, o);
         uint4* d = reinterpret_cast<uint4*>(Qs + r * pitch + 32 * u);
         d[0] = make_uint4(o[0], o[1], o[2], o[3]);
         d[1] = make_uint4(o[4], o[5], o[6], o[7]);
@@ -194,13 +195,13 @@ attention_kernel(const Params p)
         for (int it = tid; it < BN * nK16; it += THREADS) {
             const int r = it / nK16, c = it - r * nK16, j = kt * BN + r;
             cp_async16(smem_u32(rawK + (buf * BN + r) * p.raw_pitch + 16 * c),
-                       p.k + (int64_t)min(j, p.Tk - 1) * p.k_row_bytes + winK + 16 * c, j < p.Tk ? 16 : 0);
+                       p.k + (k_row0 + min(j, p.Tk - 1)) * p.k_row_bytes + winK + 16 * c, j < p.Tk ? 16 : 0);
         }
         if (with_v)
             for (int it = tid; it < BN * nV16; it += THREADS) {
                 const int r = it / nV16, c = it - r * nV16, j = kt * BN + r;
                 cp_async16(smem_u32(rawV + (buf * BN + r) * p.raw_pitch + 16 * c),
-                           p.v + (int64_t)min(j, p.Tk - 1) * p.v_row_bytes + winV + 16 * c, j < p.Tk ? 16 : 0);
+                           p.v + (k_row0 + min(j, p.Tk - 1)) * p.v_row_bytes + winV + 16 * c, j < p.Tk ? 16 : 0);
             }
         cp_async_commit();
     };
@@ -360,7 +361,7 @@ attention_kernel(const Params p)
 #pragma unroll
                             for (int e = 0; e < 4; ++e) {
                                 const int i = (e & 2) ? row1 : row0, j = kt * BN + 8 * (n + b) + 2 * t4 + (e & 1);
-                                if (i < p.Tq && j < p.Tk) p.p_dbg[((int64_t)h * p.Tq + i) * p.Tk + j] = (uint8_t)c[b][e];
+                                if (i < p.Tq && j < p.Tk) p.p_dbg[(((int64_t)blockIdx.z * p.H + h) * p.Tq + i) * p.Tk + j] = (uint8_t)c[b][e];
                             }
                     }
                 }
@@ -392,7 +393,7 @@ attention_kernel(const Params p)
                     const int pos = 32 * unit + 8 * (n & 3) + 2 * t4 + (e & 1);
                     const int i = (e & 2) ? row1 : row0;
                     if (i < p.Tq && __ldg(p.jidx_v + pos) >= 0)
-                        p.out[(int64_t)i * p.ldo + __ldg(p.src_v + pos)] = __float2half_rn(sc * (float)(O[n][e] - zv * ((e & 2) ? rs1 : rs0)));
+                        p.out[(q_row0 + i) * p.ldo + __ldg(p.src_v + pos)] = __float2half_rn(sc * (float)(O[n][e] - zv * ((e & 2) ? rs1 : rs0)));
                 }
             }
         }
@@ -427,25 +428,25 @@ static int max_units_per_head(const rptq_layout_t* L, int n_used, int H)
 }
 
 extern "C" int rptq_attention(const rptq_layout_t* LQ, const rptq_layout_t* LK, const rptq_layout_t* LV, int n_heads,
-                              const void* q_codes, int Tq, const void* k_codes, const void* v_codes, int Tk,
+                              const void* q_codes, int Tq, const void* k_codes, const void* v_codes, int Tk, int n_seq,
                               float s_P, int z_P, float qk_scale, int causal,
                               void* out_f16, int64_t ldo, uint8_t* p_codes_out, void* stream)
 {
     using namespace rptq;
     using namespace rptq::attn;
     if (!LQ || !LK || !LV || !q_codes || !k_codes || !v_codes || !out_f16) return RPTQ_ERR_INVALID_ARG;
-    if (n_heads < 1 || Tq < 0 || Tk < Tq || !(s_P > 0.f) || !(qk_scale >= 0.f)) return RPTQ_ERR_INVALID_ARG;
+    if (n_heads < 1 || Tq < 0 || Tk < Tq || n_seq < 0 || !(s_P > 0.f) || !(qk_scale >= 0.f)) return RPTQ_ERR_INVALID_ARG;
     if (LQ->g % n_heads || LK->g != LQ->g || LV->g % n_heads || ldo < LV->C) return RPTQ_ERR_INVALID_ARG;
     if (!aligned16(q_codes) || !aligned16(k_codes) || !aligned16(v_codes) || (reinterpret_cast<uintptr_t>(out_f16) & 1u)) return RPTQ_ERR_INVALID_ARG;
     // Q and K pair equal positions: same reorder index, same cluster sizes, same placement
     if (LQ->C != LK->C || LQ->size != LK->size || LQ->perm != LK->perm || LQ->pos != LK->pos || LQ->unit_cluster != LK->unit_cluster)
         return RPTQ_ERR_INVALID_ARG;
-    if (z_P != 0 || n_heads > 65535) return RPTQ_ERR_UNSUPPORTED;
+    if (z_P != 0 || n_heads > 65535 || n_seq > 65535) return RPTQ_ERR_UNSUPPORTED;
     int n_used_qk = 0, n_used_v = 0;
     if (!units_in_cluster_order(LQ, &n_used_qk) || !units_in_cluster_order(LV, &n_used_v)) return RPTQ_ERR_UNSUPPORTED;
     if (max_units_per_head(LQ, n_used_qk, n_heads) > MAX_UNITS || max_units_per_head(LV, n_used_v, n_heads) > MAX_UNITS) return RPTQ_ERR_UNSUPPORTED;
     if ((int64_t)Tk * 255 * 255 > 2147483647ll) return RPTQ_ERR_UNSUPPORTED;      // the int32 sums of the second product
-    if (Tq == 0) return RPTQ_OK;
+    if (Tq == 0 || n_seq == 0) return RPTQ_OK;
     int dev = -1;
     if (LQ->device < 0 || cudaGetDevice(&dev) != cudaSuccess) return RPTQ_ERR_CUDA;
     if (dev != LQ->device || dev != LK->device || dev != LV->device) return RPTQ_ERR_INVALID_ARG;
@@ -466,7 +467,7 @@ extern "C" int rptq_attention(const rptq_layout_t* LQ, const rptq_layout_t* LK, 
     p.raw_pitch = 4 * max_bits * MAX_UNITS + 32;          // a head's packed codes plus the alignment slack, a multiple of 16
     const int smem = (BM + BN) * QK_PITCH_MAX + 32 * V_CHUNK_UNITS * VT_PITCH + 4 * BN * p.raw_pitch;
     if (cudaFuncSetAttribute(attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return RPTQ_ERR_CUDA;
-    const dim3 grid((unsigned)((Tq + BM - 1) / BM), (unsigned)n_heads);
+    const dim3 grid((unsigned)((Tq + BM - 1) / BM), (unsigned)n_heads, (unsigned)n_seq);
     attention_kernel<<<grid, THREADS, smem, static_cast<cudaStream_t>(stream)>>>(p);
     return cudaGetLastError() == cudaSuccess ? RPTQ_OK : RPTQ_ERR_CUDA;
 }

@@ -244,3 +244,47 @@ def test_projections_write_the_cache_and_attention_reads_it():
     assert c.q.max() > 8 and c.k.max() > 8 and c.v.max() > 4          # the ranges are used
     c.qk_scale, c.s_P = 1.0 / np.sqrt(d), 1.0 / 256
     c.check(True)
+
+
+def test_several_sequences_in_one_call():
+    """Three sequences of 40 queries against 70 keys each, rows stacked: every sequence attends to its own keys only."""
+    import torch
+    from paper_2304_01089_b200 import binding
+    n_seq, Tq, Tk = 3, 40, 70
+    c = Case(31, H=2, hd=64, gh=4, Tq=n_seq * Tq, Tk=n_seq * Tk)        # the stacked tensors; the calls below see them per sequence
+    out = torch.full((n_seq * Tq, c.H * c.hd), float("nan"), dtype=torch.float16, device="cuda")
+    pc = torch.zeros((n_seq, c.H, Tq, Tk), dtype=torch.uint8, device="cuda")
+    binding.attention(c.LQ, c.LK, c.LV, c.H, c.dq, c.dk, c.dv, out, c.s_P, c.qk_scale, True, n_seq=n_seq, p_codes=pc)
+    torch.cuda.synchronize()
+    o, pq = out.float().cpu().numpy().astype(np.float64), pc.cpu().numpy()
+    ch = channel_of_oracle_position(c.perm_v, c.size_v)
+    real = ch >= 0
+    for s in range(n_seq):
+        qs, ks = slice(s * Tq, (s + 1) * Tq), slice(s * Tk, (s + 1) * Tk)
+        want, pq_want = oracle.attention(c.q[qs], c.k[ks], c.v[ks], *c.oracle_args(), True, return_p=True)
+        d = np.abs(pq[s].astype(np.int32) - pq_want.astype(np.int32))
+        assert d.max() <= 1 and (d[pq_want > 0] == 0).mean() >= 0.99
+        from_own = oracle.attention_output(pq[s], c.v[ks], c.H, c.gh, c.size_v, c.sV.astype(np.float64), c.zV, c.s_P, 0)
+        got = np.zeros_like(from_own)
+        got[:, real] = o[qs][:, ch[real]]
+        assert np.all(np.abs(got - from_own) <= 1.01 * FP16 * np.abs(from_own) + 1e-7)
+    # one sequence of the same call shape gives the same rows as the batch did
+    out1 = torch.full((Tq, c.H * c.hd), float("nan"), dtype=torch.float16, device="cuda")
+    binding.attention(c.LQ, c.LK, c.LV, c.H, c.dq[Tq:2 * Tq].contiguous(), c.dk[Tk:2 * Tk].contiguous(), c.dv[Tk:2 * Tk].contiguous(),
+                      out1, c.s_P, c.qk_scale, True)
+    torch.cuda.synchronize()
+    assert torch.equal(out1, out[Tq:2 * Tq])
+
+
+def test_empty_and_oversized_calls():
+    import torch
+    from paper_2304_01089_b200 import binding
+    c = Case(32, H=2, hd=32, gh=2, Tq=8, Tk=8)
+    out = torch.full((8, 64), 7.0, dtype=torch.float16, device="cuda")
+    binding.attention(c.LQ, c.LK, c.LV, 2, c.dq, c.dk, c.dv, out, c.s_P, c.qk_scale, True, Tq=0, Tk=8)      # no queries: nothing runs
+    binding.attention(c.LQ, c.LK, c.LV, 2, c.dq, c.dk, c.dv, out, c.s_P, c.qk_scale, True, Tq=8, Tk=8, n_seq=0)
+    torch.cuda.synchronize()
+    assert bool((out == 7.0).all())
+    with pytest.raises(binding.RptqError) as e:      # more keys than the int32 sums of the second product can take
+        binding.attention(c.LQ, c.LK, c.LV, 2, c.dq, c.dk, c.dv, out, c.s_P, c.qk_scale, True, Tq=8, Tk=40000)
+    assert e.value.status == binding.ERR_UNSUPPORTED
