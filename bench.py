@@ -51,7 +51,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             threading.Thread(target=self._read, daemon=True).start()
         except OSError:
@@ -59,9 +59,11 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append([c.strip() for c in line.split(",")])
+            self.rows.append((time.time(), [c.strip() for c in line.split(",")]))
 
-    def stop(self):
+    def stop(self, t_begin=None, t_end=None):
+        """Statistics over the samples taken between the two host times (the timed region); all samples if
+        none fall inside."""
         if self.proc is not None:
             self.proc.terminate()
             try:
@@ -70,7 +72,8 @@ class ClockSampler:
                 self.proc.kill()
         sm, mx, reasons = [], [], set()
         names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
-        for r in self.rows:
+        inside = [r for t, r in self.rows if t_begin is not None and t_begin <= t <= t_end]
+        for r in inside or [r for _, r in self.rows]:
             try:
                 sm.append(float(r[0])); mx.append(float(r[1]))
             except (ValueError, IndexError):
@@ -252,13 +255,15 @@ def run_ours(args):
     ev = [[[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in sites] for _ in range(args.steps)]
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sync_all()
+    host_begin = time.time()
     t0.record()
     for k in range(args.steps):
         _step(sites, binding, M, ev[k])
     t1.record()
     sync_all()
+    host_end = time.time()
     ms = t0.elapsed_time(t1)
-    clocks = sampler.stop()
+    clocks = sampler.stop(host_begin, host_end)
     status = binding.get_device_status()
 
     ln_ms = [[ev[k][i][0].elapsed_time(ev[k][i][1]) for k in range(args.steps)] for i in range(len(sites))]
