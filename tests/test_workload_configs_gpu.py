@@ -61,7 +61,7 @@ def _ln_codes(site, L, M):
     want_lib = np.ascontiguousarray(want[:, pos])
     got = oracle.unpack(codes[torch.from_numpy(rows).cuda()].cpu().numpy(), L.K_pad, site.bits)
     diff = np.abs(got.astype(int) - want_lib.astype(int))
-    # the benchmark spec's bar for kernel (a) against the fp64 oracle: all within +-1, >= 99.99 % equal (over the
+    # the bar of the LayerNorm kernel against the fp64 oracle: all within +-1, >= 99.99 % equal (over the
     # real positions of the sampled rows; pads always agree)
     assert diff.max() <= 1 and (diff != 0).sum() <= 1e-4 * len(rows) * site.w.hidden
     codes[torch.from_numpy(rows).cuda()] = torch.from_numpy(oracle.pack(want_lib, site.bits)).cuda()
