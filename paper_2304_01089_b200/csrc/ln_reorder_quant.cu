@@ -106,6 +106,11 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
 }
 
+// Parameters of the self-test variant only (rptq_selftest_ln_timeout sets them before its launch). They live here
+// and not in LnParams: two more fields there cost the 3-bit kernel spills in its gather loop.
+__constant__ long long c_selftest_wait_budget;     // cycles a wait may take before the block gives up
+__constant__ uint32_t c_selftest_tx_extra;         // bytes a row's barrier expects beyond what its copy delivers
+
 struct LnParams {
     const __half* x; int64_t ldx; const __half* gamma; const __half* beta; float eps;
     int M, C, n_units, n_stats_warps, depth, n_groups;
@@ -113,8 +118,6 @@ struct LnParams {
     const int32_t* jidx_tab;     // [K_pad] reordered index of each padded position, -1 at pads (debug output)
     const UnitInfo* unit_tab;
     uint8_t* codes; int64_t row_bytes; float* y_dbg; int* status;
-    long long wait_budget;       // cycles a wait may take before the block gives up
-    uint32_t tx_extra;           // self-test only: bytes a row's barrier expects beyond what its copy delivers
 };
 
 // Warp roles:
@@ -131,10 +134,14 @@ struct LnParams {
 // Per ring slot three mbarriers hand the row over: landed (copy engine) -> ready (statistics) ->
 // free (all gather warps), which lets the producer refill it.
 // DBG adds the optional fp32 output of the reordered LayerNorm values (off the fast path).
-template <int BITS, bool DBG>
+// SELFTEST: the wait budget and the extra expected bytes come from constant memory (rptq_selftest_ln_timeout);
+// otherwise they are compile-time constants.
+template <int BITS, bool DBG, bool SELFTEST = false>
 __global__ void __launch_bounds__(512)
 ln_reorder_quant_kernel(const LnParams p)
 {
+    const long long wait_budget = SELFTEST ? c_selftest_wait_budget : kLnWaitBudgetCycles;
+    const uint32_t tx_extra = SELFTEST ? c_selftest_tx_extra : 0u;
     extern __shared__ __align__(128) uint8_t smem_raw[];
     const int T = blockDim.x, C = p.C, D = p.depth, S = p.n_stats_warps;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -192,10 +199,10 @@ ln_reorder_quant_kernel(const LnParams p)
             uint32_t par = 1;                // parity to wait for on free[d]: passes at once the first time round
             for (int k = 0; k < n_rows; ++k) {
                 // the gather threads have taken their gains and biases out of the last two slots
-                if (k == D - 2) mbar_wait(bar_s + 8 * (3 * D), 0u, s_abort, p.status, p.wait_budget);
-                mbar_wait(bar_s + 8 * (2 * D + d), par, s_abort, p.status, p.wait_budget);
+                if (k == D - 2) mbar_wait(bar_s + 8 * (3 * D), 0u, s_abort, p.status, wait_budget);
+                mbar_wait(bar_s + 8 * (2 * D + d), par, s_abort, p.status, wait_budget);
                 if (*s_abort) break;         // a wait ran out somewhere in the block: issue nothing more
-                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_s + 8 * d), "r"(row_bytes_in + p.tx_extra) : "memory");
+                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_s + 8 * d), "r"(row_bytes_in + tx_extra) : "memory");
                 asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                              ::"r"(ring_s + d * pitch), "l"(src), "r"(row_bytes_in), "r"(bar_s + 8 * d) : "memory");
                 src += row_step;
@@ -208,8 +215,12 @@ ln_reorder_quant_kernel(const LnParams p)
             if (*s_abort) {
                 for (int i = n_issued > D ? n_issued - D : 0; i < n_issued; ++i) {
                     const uint32_t b = bar_s + 8 * (i % D), ph = (uint32_t)(i / D) & 1u;
-                    const long long t0 = clock64();
-                    while (!mbar_try_wait_for(b, ph, 4000u) && clock64() - t0 <= p.wait_budget) {}
+                    if constexpr (SELFTEST) {
+                        const long long t0 = clock64();
+                        while (!mbar_try_wait_for(b, ph, 4000u) && clock64() - t0 <= wait_budget) {}
+                    } else {
+                        for (int t = 0; t < (1 << 22) && !mbar_try_wait(b, ph); ++t) __nanosleep(64);
+                    }
                 }
             }
         }
@@ -228,7 +239,7 @@ ln_reorder_quant_kernel(const LnParams p)
         const uint32_t zero_s = (uint32_t)__cvta_generic_to_shared(zero16);
         for (int k = warp - 1; k < n_rows; k += S) {
             const int d = k % D;
-            mbar_wait(bar_s + 8 * d, (uint32_t)(k / D) & 1u, s_abort, p.status, p.wait_budget);
+            mbar_wait(bar_s + 8 * d, (uint32_t)(k / D) & 1u, s_abort, p.status, wait_budget);
             const uint32_t row_s = ring_s + (uint32_t)d * pitch;
             float cs[4] = {0.f, 0.f, 0.f, 0.f}, qa[4] = {0.f, 0.f, 0.f, 0.f}, qb[4] = {0.f, 0.f, 0.f, 0.f};
             const uint32_t ones = 0x3C003C00u;       // two fp16 ones
@@ -339,7 +350,7 @@ ln_reorder_quant_kernel(const LnParams p)
         uint32_t par = 0;
         for (int k = 0; k < n_rows; ++k) {
             if (turn == grp) {
-                mbar_wait(bar_s + 8 * (D + d), par, s_abort, p.status, p.wait_budget);
+                mbar_wait(bar_s + 8 * (D + d), par, s_abort, p.status, wait_budget);
                 const float2 st = stats[d];
                 const float2 rs2 = make_float2(st.x, st.x), nm2 = make_float2(st.y, st.y);
                 const uint32_t slot = (uint32_t)d * pitch;
@@ -405,6 +416,11 @@ static KernelFn pick_kernel(int bits)
 {
     return bits == 3 ? ln_reorder_quant_kernel<3, DBG> : bits == 4 ? ln_reorder_quant_kernel<4, DBG> : ln_reorder_quant_kernel<8, DBG>;
 }
+static KernelFn pick_selftest_kernel(int bits)
+{
+    return bits == 3 ? ln_reorder_quant_kernel<3, false, true> : bits == 4 ? ln_reorder_quant_kernel<4, false, true>
+                                                                           : ln_reorder_quant_kernel<8, false, true>;
+}
 
 // Launch shape of one kernel instance on one device, computed on first use (the attribute and
 // occupancy queries cost more host time than a small launch).
@@ -468,7 +484,8 @@ static int launch_ln(const rptq_layout_t* L, const void* x, int64_t ldx, const v
     if (groups > depth) groups = depth;
     const int T = 32 * (1 + S) + groups * TG;
 
-    KernelFn fn = y_dbg ? pick_kernel<true>(L->bits) : pick_kernel<false>(L->bits);
+    const bool selftest = tx_extra != 0u || wait_budget != kLnWaitBudgetCycles;
+    KernelFn fn = selftest ? pick_selftest_kernel(L->bits) : y_dbg ? pick_kernel<true>(L->bits) : pick_kernel<false>(L->bits);
     int blocks = 0;
     const int rc = planned_blocks(reinterpret_cast<const void*>(fn), dev, T, smem, &blocks);
     if (rc != RPTQ_OK) return rc;
@@ -477,7 +494,10 @@ static int launch_ln(const rptq_layout_t* L, const void* x, int64_t ldx, const v
     p.beta = static_cast<const __half*>(beta); p.eps = eps; p.M = M; p.C = C; p.n_units = L->n_units;
     p.n_stats_warps = S; p.depth = depth; p.n_groups = groups; p.ch_tab = L->d_src; p.jidx_tab = L->d_jidx; p.unit_tab = L->d_unit;
     p.codes = static_cast<uint8_t*>(codes); p.row_bytes = L->row_bytes; p.y_dbg = y_dbg; p.status = device_status_word();
-    p.wait_budget = wait_budget; p.tx_extra = tx_extra;
+    if (selftest) {
+        if (cudaMemcpyToSymbol(c_selftest_wait_budget, &wait_budget, sizeof(wait_budget)) != cudaSuccess ||
+            cudaMemcpyToSymbol(c_selftest_tx_extra, &tx_extra, sizeof(tx_extra)) != cudaSuccess) return RPTQ_ERR_CUDA;
+    }
     fn<<<M < blocks ? M : blocks, T, smem, static_cast<cudaStream_t>(stream)>>>(p);
     return cudaGetLastError() == cudaSuccess ? RPTQ_OK : RPTQ_ERR_CUDA;
 }
