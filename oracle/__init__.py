@@ -339,6 +339,27 @@ def attention(q_codes, k_codes, v_codes, H: int, gh: int, size_qk, sQ, zQ, sK, z
     return (out, pq) if return_p else out
 
 
+def attention_kv(q, ch_of_pos_k, k_codes, v_codes, H: int, gh: int, size_k, sK, zK, size_v, sV, zV,
+                 qk_scale: float, causal: bool) -> np.ndarray:
+    """Sec. 5.2, key / value cache quantised only: q [Tq][C] floating point in the original channel order,
+    ch_of_pos_k int [K_pad_k] the channel at each padded position of K's layout (-1 at pads), codes at
+    padded positions. Returns O [Tq][K_pad_v]."""
+    q = _arr(q, np.float64)
+    ch = _arr(ch_of_pos_k, np.int32)
+    k_codes, v_codes = _arr(k_codes, np.uint8), _arr(v_codes, np.uint8)
+    size_k, size_v = _arr(size_k, np.int32), _arr(size_v, np.int32)
+    sK, sV, zK, zV = _arr(sK, np.float64), _arr(sV, np.float64), _arr(zK, np.int32), _arr(zV, np.int32)
+    Tq, Cn = q.shape
+    Tk, kpk = k_codes.shape
+    kpv = v_codes.shape[1]
+    assert ch.shape == (kpk,) and v_codes.shape[0] == Tk and Tq <= Tk and size_k.shape == (H * gh,) == size_v.shape
+    out = np.empty((Tq, kpv))
+    _lib.orc_attention_kv(_p(q), C.c_int(Cn), _p(ch), _p(k_codes), _p(v_codes), _i64(Tq), _i64(Tk), C.c_int(H), C.c_int(gh),
+                          _i32(kpk), _p(size_k), _p(sK), _p(zK), _i32(kpv), _p(size_v), _p(sV), _p(zV),
+                          _dbl(qk_scale), C.c_int(1 if causal else 0), _p(out))
+    return out
+
+
 def attention_output(p_codes, v_codes, H: int, gh: int, size_v, sV, zV, s_P: float, z_P: int) -> np.ndarray:
     """O from given softmax codes p_codes [H][Tq][Tk] and V codes [Tk][K_pad_v]."""
     p_codes, v_codes = _arr(p_codes, np.uint8), _arr(v_codes, np.uint8)

@@ -840,3 +840,53 @@ void orc_attention_output(const uint8_t* p_codes, const uint8_t* v_codes, int64_
                 }
     free(off_v);
 }
+
+/* Sec. 5.2, the schemes that quantise only the key / value cache (W4A4KV, W4A3KV, W3A3KV): the query
+ * and the softmax output stay 16-bit floating point, the cached keys and values are per-cluster codes
+ * of the per-head layouts. Attention as its definition on the de-quantised cache:
+ *   K^[j][ch] = sK_c (Kq - zK_c), V^ likewise;  A[i][j] = qk_scale * sum over the head's channels of Q[i][ch] K^[j][ch];
+ *   visibility as in orc_attention;  P = softmax over the visible keys;  O[i][p] = sum_j P[i][j] V^[j][p].
+ * q is [Tq][C] in the ORIGINAL channel order (head h owns channels h * C / H ..); ch_of_pos_k[K_pad_k]
+ * gives the channel at each padded position of K's layout (-1 at pads). out is [Tq][K_pad_v], 0 at pads.
+ * Nothing is rounded here: the 16-bit roundings of an implementation are the caller's tolerance. */
+void orc_attention_kv(const double* q, int C, const int32_t* ch_of_pos_k, const uint8_t* k_codes, const uint8_t* v_codes,
+                      int64_t Tq, int64_t Tk, int H, int gh,
+                      int32_t K_pad_k, const int32_t* size_k, const double* sK, const int32_t* zK,
+                      int32_t K_pad_v, const int32_t* size_v, const double* sV, const int32_t* zV,
+                      double qk_scale, int causal, double* out)
+{
+    const int g = H * gh;
+    int32_t* off_k = (int32_t*)malloc(sizeof(int32_t) * (g + 1));
+    int32_t* off_v = (int32_t*)malloc(sizeof(int32_t) * (g + 1));
+    orc_segment_offsets(size_k, g, off_k);
+    orc_segment_offsets(size_v, g, off_v);
+    memset(out, 0, sizeof(double) * (size_t)Tq * (size_t)K_pad_v);
+#pragma omp parallel for schedule(dynamic, 4) collapse(2)
+    for (int h = 0; h < H; ++h)
+        for (int64_t i = 0; i < Tq; ++i) {
+            double* A = (double*)malloc(sizeof(double) * (size_t)Tk);
+            const int64_t last = causal ? i + (Tk - Tq) : Tk - 1;
+            double top = -INFINITY;
+            for (int64_t j = 0; j <= last; ++j) {
+                double a = 0.0;
+                for (int c = h * gh; c < (h + 1) * gh; ++c)
+                    for (int p = off_k[c]; p < off_k[c] + size_k[c]; ++p)
+                        a += q[i * C + ch_of_pos_k[p]] * (sK[c] * ((double)k_codes[j * K_pad_k + p] - (double)zK[c]));
+                A[j] = qk_scale * a;
+                if (A[j] > top) top = A[j];
+            }
+            double denom = 0.0;
+            for (int64_t j = 0; j <= last; ++j) denom += exp(A[j] - top);
+            for (int64_t j = 0; j < Tk; ++j) A[j] = j <= last ? exp(A[j] - top) / denom : 0.0;
+            for (int c = h * gh; c < (h + 1) * gh; ++c)
+                for (int p = off_v[c]; p < off_v[c] + size_v[c]; ++p) {
+                    double o = 0.0;
+                    for (int64_t j = 0; j < Tk; ++j)
+                        o += A[j] * (sV[c] * ((double)v_codes[j * K_pad_v + p] - (double)zV[c]));
+                    out[i * K_pad_v + p] = o;
+                }
+            free(A);
+        }
+    free(off_k);
+    free(off_v);
+}

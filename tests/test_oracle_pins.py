@@ -606,6 +606,8 @@ def test_attention_hand_worked_example():
     n = 0
     for line in _golden_rows("attention_toy.txt"):
         kind, pq_want, o_want = [p.strip() for p in line.split("|")]
+        if kind.startswith("kv_"):
+            continue
         o, pq = _toy_attention(kind == "causal")
         assert pq.reshape(-1).tolist() == [int(t) for t in pq_want.split()]
         got = np.concatenate([o[:, 0:1], o[:, 32:34]], axis=1).reshape(-1)
@@ -709,3 +711,57 @@ def test_attention_closed_forms():
         vlo, vhi = c["off_v"][h * gh], c["off_v"][(h + 1) * gh]
         assert np.allclose(o[:, vlo:vhi], (255.0 / 256) * Vh[best, vlo:vhi], rtol=0, atol=1e-12)
         assert np.all(pq[h][np.arange(4), best] == 255) and pq[h].sum() == 4 * 255
+
+
+def _toy_kv_inputs():
+    k = np.zeros((2, 128), np.uint8); v = np.zeros((2, 128), np.uint8)
+    k[0, 0:2] = (2, 3); k[0, 32] = 5; k[1, 0:2] = (3, 1); k[1, 32] = 3
+    v[0, 0] = 8; v[0, 32:34] = (3, 0); v[1, 0] = 0; v[1, 32:34] = (1, 2)
+    ch = np.full(128, -1, np.int32); ch[0:2] = (2, 0); ch[32] = 1            # K's positions hold channels 2, 0 | 1
+    q = np.zeros((2, 3)); q[0, [2, 0, 1]] = (1, 0, 2); q[1, [2, 0, 1]] = (2, -1, 2)
+    return q, ch, k, v
+
+
+def test_kv_only_attention_hand_worked_example():
+    n = 0
+    for line in _golden_rows("attention_toy.txt"):
+        kind, _, o_want = [p.strip() for p in line.split("|")]
+        if not kind.startswith("kv_"):
+            continue
+        q, ch, k, v = _toy_kv_inputs()
+        o = oracle.attention_kv(q, ch, k, v, 1, 2, [2, 1], [1.0, 0.5], [1, 3], [1, 2], [0.25, 2.0], [4, 1], np.log(3.0) / 2, kind == "kv_causal")
+        got = np.concatenate([o[:, 0:1], o[:, 32:34]], axis=1).reshape(-1)
+        assert np.allclose(got, [float(t) for t in o_want.split()], rtol=0, atol=1e-14)
+        assert not o[:, 1:32].any() and not o[:, 34:].any()
+        n += 1
+    assert n == 2
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_kv_only_attention_is_plain_attention_on_the_dequantised_cache(causal):
+    """The definition itself, through library routines: scipy softmax and numpy matmul on K^, V^ de-quantised by hand,
+    with the query's channels scattered over K's positions."""
+    from scipy.special import softmax
+    for seed in (4, 5):
+        c = _attention_case(seed)
+        r = _rng(100 + seed)
+        Tq, Tk, H, gh, hd = c["q"].shape[0], c["k"].shape[0], c["H"], c["gh"], c["hd"]
+        Cn = H * hd
+        k_pad = c["k"].shape[1]
+        ch = np.full(k_pad, -1, np.int32)                       # a random per-head assignment of channels to K's real positions
+        for h in range(H):
+            pos = np.concatenate([np.arange(c["off_qk"][cc], c["off_qk"][cc] + c["size_qk"][cc]) for cc in range(h * gh, (h + 1) * gh)])
+            ch[pos] = h * hd + r.permutation(hd)
+        q = r.normal(size=(Tq, Cn))
+        scale = 1.0 / np.sqrt(hd)
+        o = oracle.attention_kv(q, ch, c["k"], c["v"], H, gh, c["size_qk"], c["sK"], c["zK"], c["size_v"], c["sV"], c["zV"], scale, causal)
+        Kh = _dequant_by_hand(c["k"], c["off_qk"], c["size_qk"], c["sK"], c["zK"])
+        Vh = _dequant_by_hand(c["v"], c["off_v"], c["size_v"], c["sV"], c["zV"])
+        for h in range(H):
+            lo, hi = c["off_qk"][h * gh], c["off_qk"][(h + 1) * gh]
+            real = ch[lo:hi] >= 0
+            A = scale * q[:, ch[lo:hi][real]] @ Kh[:, lo:hi][:, real].T
+            if causal:
+                A = np.where(np.arange(Tk)[None, :] <= np.arange(Tq)[:, None] + (Tk - Tq), A, -np.inf)
+            vlo, vhi = c["off_v"][h * gh], c["off_v"][(h + 1) * gh]
+            assert np.allclose(o[:, vlo:vhi], softmax(A, axis=1) @ Vh[:, vlo:vhi], rtol=1e-12, atol=1e-12)
