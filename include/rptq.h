@@ -374,6 +374,24 @@ int rptq_attention(const rptq_layout_t* LQ, const rptq_layout_t* LK, const rptq_
                    float s_P, int z_P, float qk_scale, int causal,
                    void* out_f16, int64_t ldo, uint8_t* p_codes_out, void* stream);
 
+/*
+ * Sec. 5.2, the schemes that quantise only the key / value cache (W4A4KV, W4A3KV, W3A3KV): the query and
+ * the softmax output stay 16-bit floating point; the cached keys and values are per-cluster codes of the
+ * per-head layouts LK and LV (as for rptq_attention; K's layout is the one Q and K were clustered for). For
+ * head h, query i, key j:
+ *   A[i][j]  = qk_scale * sum_c s^K_c sum_{p in c} Q[i][ch(p)] (K_q[j][p] - z^K_c)     ch(p): the channel at K's position p
+ *   P        = softmax of A over the visible keys (as for rptq_attention), fp32, rounded to fp16 for the second product
+ *   O[i][ch] = s^V_c (sum_j P[i][j] V_q[j][p] / sum_j P[i][j] - z^V_c)                 fp16
+ * fp16 x fp16 products with fp32 sums on the tensor cores (the codes are exact in fp16).
+ *   q_f16    dev fp16 [n_seq * Tq][ldq], ldq >= C, original channel order (head h owns channels h * C / n_heads ..)
+ *   k_codes, v_codes  dev, n_seq * Tk rows of LK.row_bytes / LV.row_bytes bytes
+ *   out_f16  dev fp16 [n_seq * Tq][ldo], ldo >= C, original channel order
+ * Limits as for rptq_attention (eight units per head and layout, Tk >= Tq, n_seq, n_heads <= 65535).
+ */
+int rptq_attention_kv(const rptq_layout_t* LK, const rptq_layout_t* LV, int n_heads,
+                      const void* q_f16, int64_t ldq, int Tq, const void* k_codes, const void* v_codes, int Tk, int n_seq,
+                      float qk_scale, int causal, void* out_f16, int64_t ldo, void* stream);
+
 const char* rptq_status_string(int status);
 int rptq_format_version(void);
 

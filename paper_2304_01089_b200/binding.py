@@ -28,7 +28,7 @@ EXPORTS = (
     "rptq_format_version", "rptq_layout_padded_index", "rptq_weight_codes_bytes", "rptq_cluster_gemm_noalloc",
     "rptq_selftest_ln_timeout", "rptq_dequant_gemm", "rptq_ln_channel_minmax", "rptq_kmeans", "rptq_kmeans_workspace_bytes",
     "rptq_probe_int8_peak", "rptq_weight_pack_clustered", "rptq_code_rowsums", "rptq_cluster_gemm_clustered",
-    "rptq_attention",
+    "rptq_attention", "rptq_attention_kv",
 )
 
 
@@ -71,6 +71,7 @@ def _load(path: str = LIB_PATH) -> C.CDLL:
     lib.rptq_status_string.argtypes = [i32]
     lib.rptq_status_string.restype = C.c_char_p
     lib.rptq_attention.argtypes = [vp, vp, vp, i32, vp, i32, vp, vp, i32, i32, f32, i32, f32, i32, vp, i64, vp, vp]
+    lib.rptq_attention_kv.argtypes = [vp, vp, i32, vp, i64, i32, vp, vp, i32, i32, f32, i32, vp, i64, vp]
     for name in EXPORTS:
         if name not in ("rptq_status_string", "rptq_weight_codes_bytes", "rptq_kmeans_workspace_bytes"):
             getattr(lib, name).restype = i32
@@ -218,6 +219,17 @@ def attention(LQ: Layout, LK: Layout, LV: Layout, n_heads: int, q_codes, k_codes
     _check(_lib.rptq_attention(LQ.handle, LK.handle, LV.handle, int(n_heads), _dev_ptr(q_codes), Tq, _dev_ptr(k_codes),
                                _dev_ptr(v_codes), Tk, int(n_seq), C.c_float(s_P), int(z_P), C.c_float(qk_scale), 1 if causal else 0,
                                _dev_ptr(out), int(out.stride(0)), _dev_ptr(p_codes), _stream_ptr(stream)), "rptq_attention")
+
+
+def attention_kv(LK: Layout, LV: Layout, n_heads: int, q, k_codes, v_codes, out, qk_scale: float, causal: bool,
+                 Tq: Optional[int] = None, Tk: Optional[int] = None, n_seq: int = 1, stream=None) -> None:
+    """rptq_attention_kv: q fp16 [n_seq * Tq][>= C] (original channel order), k_codes / v_codes uint8
+    [n_seq * Tk][row_bytes], out fp16 [n_seq * Tq][>= C]: CUDA tensors."""
+    Tq = int(q.shape[0]) // int(n_seq) if Tq is None else int(Tq)
+    Tk = int(k_codes.shape[0]) // int(n_seq) if Tk is None else int(Tk)
+    _check(_lib.rptq_attention_kv(LK.handle, LV.handle, int(n_heads), _dev_ptr(q), int(q.stride(0)), Tq, _dev_ptr(k_codes),
+                                  _dev_ptr(v_codes), Tk, int(n_seq), C.c_float(qk_scale), 1 if causal else 0,
+                                  _dev_ptr(out), int(out.stride(0)), _stream_ptr(stream)), "rptq_attention_kv")
 
 
 def weight_pack(layout_in: Layout, W: np.ndarray, out_perm=None, n_pad: Optional[int] = None):
