@@ -168,8 +168,22 @@ def _attention_leg(w, M, torch, binding):
     torch.cuda.synchronize()
     us = float(np.median([ev[i].elapsed_time(ev[i + 1]) for i in range(n_rep)])) * 1e3
     ops = 2.0 * n_seq * H * (T * (T + 1) / 2) * 128 * 2    # both products once, visible keys, real channels
+    # the same cache read by a 16-bit query (only the key / value cache quantised)
+    q16 = torch.randn((n_seq * T, w.hidden), dtype=torch.float16, device="cuda", generator=torch.Generator(device="cuda").manual_seed(w.seed))
+    run_kv = lambda: binding.attention_kv(LK, LV, H, q16, dev[1], dev[2], out, 1.0 / np.sqrt(128.0), True, n_seq=n_seq)
+    for _ in range(3):
+        run_kv()
+    torch.cuda.synchronize()
+    for i in range(n_rep):
+        ev[i].record()
+        run_kv()
+    ev[n_rep].record()
+    torch.cuda.synchronize()
+    us_kv = float(np.median([ev[i].elapsed_time(ev[i + 1]) for i in range(n_rep)])) * 1e3
     return {"kernel": "attention_kernel", "heads": H, "head_dim": 128, "clusters_per_head": 4, "sequences": n_seq, "tokens": T, "causal": True,
             "bits": w.bits, "us": us, "TOPS": ops / us / 1e6,
+            "kv_only": {"kernel": "attention_kv_kernel", "us": us_kv, "TFLOPS": ops / us_kv / 1e6,
+                        "note": "16-bit query and probabilities, quantised key / value cache; fp16 mma.sync m16n8k16"},
             "note": "integer products on mma.sync m16n8k32 (the scores are computed twice: the softmax codes need the finished row sums)"}
 
 

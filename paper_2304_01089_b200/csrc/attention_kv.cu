@@ -228,9 +228,11 @@ attention_kv_kernel(const Params p)
         const float r0 = ex2(m0 - n0), r1 = ex2(m1 - n1);    // what the sums so far shrink by
         m0 = n0; m1 = n1;
         l0 *= r0; l1 *= r1;
+        if (__any_sync(0xffffffffu, r0 != 1.f || r1 != 1.f)) {       // a row maximum of this warp moved (rare after the first tiles)
 #pragma unroll
-        for (int n = 0; n < 4 * MAX_UNITS; ++n) {
-            if (n < 4 * nuv) { O[n][0] *= r0; O[n][1] *= r0; O[n][2] *= r1; O[n][3] *= r1; }
+            for (int n = 0; n < 4 * MAX_UNITS; ++n) {
+                if (n < 4 * nuv) { O[n][0] *= r0; O[n][1] *= r0; O[n][2] *= r1; O[n][3] *= r1; }
+            }
         }
         // probabilities (not normalised) as fp16, in the layout of the second product's first operand; the row
         // sums add the rounded values, so that the division at the end normalises exactly what was multiplied
