@@ -144,12 +144,24 @@ attention_kv_kernel(const Params p)
         s_coef[tid] = __ldg(&p.unit_sz_k[uk0 + tid].x) * p.qk_scale_log2e;
         s_last[tid] = (tid == nuk - 1) || (__ldg(p.unit_cluster_k + uk0 + tid + 1) != __ldg(p.unit_cluster_k + uk0 + tid));
     }
-    // the queries' channels in K's position order (pads 0)
-    for (int it = tid; it < BM * 32 * nuk; it += THREADS) {
-        const int r = it / (32 * nuk), pp = it - r * (32 * nuk), pos = 32 * uk0 + pp;
+    // The queries' channels in K's position order (pads 0): the head's slice of every row is read in memory order
+    // (independent, coalesced loads) into the K tile's buffer, then permuted from there.
+    __shared__ int16_t s_chan[32 * MAX_UNITS];               // channel within the head at each of its positions, -1 at pads
+    for (int pp = tid; pp < 32 * nuk; pp += THREADS) {
+        const int pos = 32 * uk0 + pp;
+        s_chan[pp] = __ldg(p.jidx_k + pos) >= 0 ? (int16_t)((int)__ldg(p.src_k + pos) - h * p.hd) : (int16_t)-1;
+    }
+    for (int it = tid; it < BM * p.hd; it += THREADS) {
+        const int r = it / p.hd, c = it - r * p.hd;
         __half v = __float2half_rn(0.f);
-        if (i0 + r < p.Tq && __ldg(p.jidx_k + pos) >= 0) v = p.q[(q_row0 + i0 + r) * p.ldq + __ldg(p.src_k + pos)];
-        *reinterpret_cast<__half*>(Qs + r * PITCH + 2 * pp) = v;
+        if (i0 + r < p.Tq) v = p.q[(q_row0 + i0 + r) * p.ldq + h * p.hd + c];
+        *reinterpret_cast<__half*>(Ks + r * PITCH + 2 * c) = v;
+    }
+    __syncthreads();
+    for (int it = tid; it < BM * 32 * nuk; it += THREADS) {
+        const int r = it / (32 * nuk), pp = it - r * (32 * nuk);
+        const int c = s_chan[pp];
+        *reinterpret_cast<__half*>(Qs + r * PITCH + 2 * pp) = c >= 0 ? *reinterpret_cast<const __half*>(Ks + r * PITCH + 2 * c) : __float2half_rn(0.f);
     }
     __syncthreads();
 
@@ -302,6 +314,17 @@ static bool kv_units_in_cluster_order(const rptq_layout_t* L, int* n_used)
     return true;
 }
 
+// head h's clusters hold exactly the channels h * hd .. (h + 1) * hd - 1 (the kernel reads a head's query slice by that rule)
+static bool kv_heads_own_their_channels(const rptq_layout_t* L, int H)
+{
+    const int gh = L->g / H, hd = L->C / H;
+    size_t j = 0;
+    for (int c = 0; c < L->g; ++c)
+        for (int i = 0; i < L->size[(size_t)c]; ++i, ++j)
+            if (L->perm[j] / hd != c / gh) return false;
+    return true;
+}
+
 static int kv_max_units_per_head(const rptq_layout_t* L, int n_used, int H)
 {
     const int gh = L->g / H;
@@ -327,6 +350,7 @@ extern "C" int rptq_attention_kv(const rptq_layout_t* LK, const rptq_layout_t* L
     int n_used_k = 0, n_used_v = 0;
     if (!kv_units_in_cluster_order(LK, &n_used_k) || !kv_units_in_cluster_order(LV, &n_used_v)) return RPTQ_ERR_UNSUPPORTED;
     if (kv_max_units_per_head(LK, n_used_k, n_heads) > MAX_UNITS || kv_max_units_per_head(LV, n_used_v, n_heads) > MAX_UNITS) return RPTQ_ERR_UNSUPPORTED;
+    if (!kv_heads_own_their_channels(LK, n_heads)) return RPTQ_ERR_INVALID_ARG;
     if (Tq == 0 || n_seq == 0) return RPTQ_OK;
     int dev = -1;
     if (LK->device < 0 || cudaGetDevice(&dev) != cudaSuccess) return RPTQ_ERR_CUDA;

@@ -110,6 +110,20 @@ def test_refusals_and_empty_calls():
     assert e.value.status == binding.ERR_INVALID_ARG
 
 
+def test_layouts_whose_heads_do_not_own_their_channels_are_refused():
+    import torch
+    from paper_2304_01089_b200 import binding
+    from helpers import random_layout_params
+    rng = np.random.default_rng(9)
+    perm, size, scale, zero = random_layout_params(rng, 64, 4, 4, allow_empty=False)     # one permutation across both heads
+    L = binding.Layout(perm, size, scale, zero, 4)
+    q = torch.zeros((8, 64), dtype=torch.float16, device="cuda")
+    codes = torch.zeros((8, L.row_bytes), dtype=torch.uint8, device="cuda")
+    with pytest.raises(binding.RptqError) as e:
+        binding.attention_kv(L, L, 2, q, codes, codes, torch.zeros_like(q), 0.1, True)
+    assert e.value.status == binding.ERR_INVALID_ARG
+
+
 def test_opt66b_heads_sampled_rows():
     """72 heads of 128 channels, 2048 tokens, 4-bit cache, causal; sampled (head, query) rows against the oracle
     run on that head and that query alone."""
